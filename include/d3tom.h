@@ -1,0 +1,191 @@
+/*
+ * d3tom.h -- C ABI of the D3ToM merge-layer library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the merge-layer work of ONE denoising step of a
+ * diffusion multimodal LLM with decider-guided token merging:
+ *
+ *   d3tom_attn_importance   bidirectional self-attention at the merge layer l*
+ *                           + the decider->visual importance map, one pass
+ *   d3tom_select            keep / merge partition by rank of the importance
+ *   d3tom_merge             nearest-kept-neighbour routing by cosine similarity,
+ *                           aggregation, physical removal of the merged rows
+ *   d3tom_attn_varlen       bidirectional attention over the shortened sequences
+ *   d3tom_proj_qkv          (supporting) Q,K,V projection of a post-merge layer
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - A batch holds B requests packed back to back.  Request b is the
+ *    concatenation [visual | prompt | response] (Algorithm 1, Embed(Concat(V,P,X)))
+ *    and occupies packed rows [cu_seqlens[b], cu_seqlens[b+1]); its first
+ *    n_visual[b] rows are the visual tokens.
+ *  - Activations are row-major [rows, H, dh] == [rows, D], D = H*dh, in the
+ *    storage type `dt` (bf16 or fp32).
+ *  - Unless a parameter says "host", every pointer is DEVICE memory owned by
+ *    the caller and valid on the context's device.  The library never
+ *    allocates, frees or resizes caller buffers, never synchronises the
+ *    stream and never changes the current device; all work is enqueued on
+ *    `stream` and is complete when the stream reaches that point.
+ *  - Scratch memory lives in the context and is sized once, at
+ *    d3tom_create, from d3tom_limits.  A call that needs more returns
+ *    D3TOM_ERR_WORKSPACE; nothing is reallocated.  Two calls on the same
+ *    context must not overlap on the GPU (use one context per stream).
+ *  - Every function returns a status: D3TOM_OK (0) or a negative error.  No
+ *    exceptions, no abort, nothing printed.  Argument errors are detected on
+ *    the host before anything is launched.  Problems only the device can see
+ *    (a bounded wait that ran out) are recorded in a status word read by
+ *    d3tom_device_status.
+ *  - bf16 runs on the tcgen05 tensor-core kernels and needs head_dim 64 or
+ *    128; fp32 runs on plain CUDA-core kernels (any head_dim that is a
+ *    multiple of 4 up to 128).  There is no CPU fallback.
+ */
+#ifndef D3TOM_H_
+#define D3TOM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct d3tom_ctx d3tom_ctx;          /* opaque; owns scratch only */
+typedef void* d3tom_stream;                  /* a cudaStream_t */
+
+typedef enum { D3TOM_BF16 = 0, D3TOM_FP32 = 1 } d3tom_dtype;
+typedef enum { D3TOM_AGG_SUM = 0, D3TOM_AGG_MEAN = 1 } d3tom_agg;
+
+enum {
+  D3TOM_OK = 0,
+  D3TOM_ERR_INVALID_ARG = -1,   /* null pointer, negative size, inconsistent sizes */
+  D3TOM_ERR_UNSUPPORTED = -2,   /* dtype / head_dim / device architecture not supported */
+  D3TOM_ERR_WORKSPACE   = -3,   /* request exceeds the limits given at d3tom_create */
+  D3TOM_ERR_CUDA        = -4,   /* a CUDA runtime / driver call failed (see d3tom_last_cuda_error) */
+  D3TOM_ERR_TIMEOUT     = -5    /* device status: a bounded wait inside a kernel ran out */
+};
+
+typedef struct {
+  int max_total_tokens;        /* packed rows over the whole batch */
+  int max_batch;               /* requests per call */
+  int heads;                   /* H */
+  int head_dim;                /* dh */
+  int max_deciders;            /* decider tokens over the whole batch */
+  int max_visual_per_request;  /* largest n_visual[b] */
+} d3tom_limits;
+
+/* Create a context on CUDA device `device` (must be sm_100) and allocate its
+ * scratch.  Returns D3TOM_ERR_UNSUPPORTED on any other architecture. */
+int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim);
+int d3tom_destroy(d3tom_ctx* ctx);
+const char* d3tom_status_string(int status);
+/* cudaError_t / CUresult of the last failing CUDA call on this context (0 if none). */
+int d3tom_last_cuda_error(const d3tom_ctx* ctx);
+/* Copies the device-side status word to *status_out (host).  Synchronises the
+ * device; call it after the stream work of interest has been waited for. */
+int d3tom_device_status(d3tom_ctx* ctx, int* status_out);
+/* Bytes of scratch the context holds (host query). */
+int64_t d3tom_workspace_bytes(const d3tom_ctx* ctx);
+
+/* Debugging aid: with on != 0, bf16 calls also run on the plain CUDA-core
+ * kernels that serve fp32 (slow; lets the two code paths be compared on the GPU). */
+int d3tom_set_reference_kernels(d3tom_ctx* ctx, int on);
+
+/* Sec. 3.2.1, "Rank(S_j) <= (1-alpha)|V|": number of kept tokens for keep
+ * ratio r = 1-alpha.  Host arithmetic: clamp(floor(r*n_visual + 1e-9), 1, n_visual). */
+int d3tom_keep_count(int n_visual, double keep_ratio);
+
+/* Sec. 3.2.3, linear schedule: alpha at decode-order step `step` in 0..T-1 is
+ * a_min + (a_max - a_min) * step/(T-1) (smallest at the beginning of decoding);
+ * `reversed` != 0 gives the high->low ablation.  Host arithmetic. */
+int d3tom_schedule_alpha(int step, int T, double a_min, double a_max, int reversed, double* alpha_out);
+
+/* Sec. 3.2.1 (self-attention matrix A and decider score S_j); Algorithm 1,
+ * SelfAttn_l and the line S_j <- sum_{i in D} A_ij.
+ *
+ * Per request and head: O = softmax(Q K^T * softmax_scale) V over ALL keys of
+ * the request (no mask).  In the same pass, for every visual key j,
+ *   importance[cu_vis[b] + j] = sum over heads, sum over decider rows i of A_ij.
+ *
+ *  q, k, v       [total, H, dh] storage type
+ *  cu_seqlens    [B+1] int32, n_visual [B] int32
+ *  decider_pos   [cu_deciders[B]] int32: decider rows relative to the request
+ *                start, strictly ascending per request
+ *  cu_deciders   [B+1] int32.  A request with no deciders gets importance 0.
+ *  n_deciders_total  == cu_deciders[B] (host copy, sizes the scratch use)
+ *  total_tokens  == cu_seqlens[B]; max_seqlen >= every request length;
+ *  max_visual >= every n_visual[b] (host copies)
+ *  attn_out      [total, H*dh] storage type (the post-attention states H~)
+ *  importance    [cu_vis[B]] fp32, cu_vis [B+1] int32
+ * The importance is reduced in a fixed order: results are run-to-run identical. */
+int d3tom_attn_importance(d3tom_ctx* ctx, d3tom_dtype dt,
+                          const void* q, const void* k, const void* v,
+                          const int32_t* cu_seqlens, const int32_t* n_visual,
+                          const int32_t* decider_pos, const int32_t* cu_deciders,
+                          int B, int total_tokens, int max_seqlen, int max_visual, int n_deciders_total,
+                          float softmax_scale,
+                          void* attn_out, float* importance, const int32_t* cu_vis,
+                          d3tom_stream stream);
+
+/* Sec. 3.2.1, the partition V_kept / V_merge; Algorithm 1, TopK.
+ *
+ * Per request: the keep_count[b] visual tokens of highest importance, ordered by
+ * (score descending, index ascending) on the fp32 bit pattern, emitted
+ * ASCENDING by position.
+ *  importance  [cu_vis[B]] fp32 (finite, >= 0)
+ *  keep_count  [B] int32, 1 <= keep_count[b] <= n_visual[b]
+ *  cu_kept     [B+1] int32, prefix sum of keep_count
+ *  kept_idx    [cu_kept[B]] int32 out: positions relative to the request start
+ *  keep_mask   [cu_vis[B]] uint8 out: 1 = kept, 0 = merged away
+ *  max_visual  host: >= every n_visual[b] */
+int d3tom_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis,
+                 const int32_t* keep_count, const int32_t* cu_kept, int B, int max_visual,
+                 int32_t* kept_idx, uint8_t* keep_mask, d3tom_stream stream);
+
+/* Sec. 3.2.2 (similarity-based merging); Algorithm 1, the loop over V_merge
+ * and the removal of the merged positions.
+ *
+ * For every pruned visual token m: k* = argmax over the request's kept tokens
+ * of cos(h~_m, h~_k), cosines taken on the PRE-merge states in fp32
+ * (dot * (1/|h_m|) * (1/|h_k|), zero-norm rows give 0), ties to the lowest kept
+ * position.  Then out_k = h~_k + sum of its members (SUM, the paper's
+ * equation) or that divided by 1 + members (MEAN), accumulated in fp32 in
+ * ascending member order and rounded once.  The output sequence of request b
+ * is [merged kept visual rows, ascending position | prompt | response].
+ *
+ *  hidden          [total_tokens, D] storage type
+ *  kept_idx/cu_kept  from d3tom_select
+ *  total_out       host: sum over b of N_b - n_visual[b] + k_b  (== cu_seqlens_out[B])
+ *  max_visual, max_kept  host: >= every n_visual[b] / keep count
+ *  hidden_out      [total_out, D] out
+ *  cu_seqlens_out  [B+1] int32 in: prefix sum of the shortened lengths (host-computed by the caller)
+ *  assign          [cu_vis[B]] int32 out: destination slot (rank in the kept list) of every visual token
+ *  member_count    [cu_kept[B]] int32 out: pruned tokens routed to each kept token
+ *  src_of_dst      [total_out] int32 out: original packed row of every output row
+ *  sim_debug       nullable; [cu_vis[B], max_kept] fp32 out: entry (cu_vis[b]+m, s) is the
+ *                  cosine of pruned token m with the kept token of slot s, exactly the
+ *                  value the argmax compared; rows of kept tokens are not written */
+int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode,
+                const void* hidden, const int32_t* cu_seqlens, const int32_t* n_visual, const int32_t* cu_vis,
+                const int32_t* kept_idx, const int32_t* cu_kept,
+                int B, int D, int total_tokens, int total_out, int max_visual, int max_kept,
+                void* hidden_out, const int32_t* cu_seqlens_out,
+                int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
+                float* sim_debug, d3tom_stream stream);
+
+/* Sec. 3.2.2, last paragraph: the layers after l* run on the shortened tensor.
+ * Same attention as d3tom_attn_importance, over packed ragged sequences, with
+ * no importance output. */
+int d3tom_attn_varlen(d3tom_ctx* ctx, d3tom_dtype dt,
+                      const void* q, const void* k, const void* v,
+                      const int32_t* cu_seqlens, int B, int total_tokens, int max_seqlen,
+                      float softmax_scale, void* out, d3tom_stream stream);
+
+/* Sec. 3.2.1, Q = H W_Q, K = H W_K (and V): the projection feeding a
+ * post-merge layer.  x [total, D]; w_qkv [3D, D] row-major, row o holds the
+ * weights of output feature o (rows 0..D-1 -> Q, D..2D-1 -> K, 2D..3D-1 -> V);
+ * q, k, v [total, D] out, fp32 accumulation, one rounding to the storage type. */
+int d3tom_proj_qkv(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_qkv,
+                   int total, int D, void* q, void* k, void* v, d3tom_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D3TOM_H_ */

@@ -1,0 +1,265 @@
+// bf16 x bf16 -> fp32 "NT" GEMM on tcgen05 tensor cores, C[m, n] = sum_k A[m, k] B[n, k],
+// with two fused epilogues:
+//
+//   kEpiProj  the Q,K,V projection of a post-merge layer (Sec. 3.2.1, Q = H W_Q,
+//             K = H W_K): rounds to bf16 and writes the tile into q, k or v.
+//   kEpiSim   the similarity step of the merge (Sec. 3.2.2, arg max of the cosine
+//             over the kept set): scales the dot products by the two inverse norms
+//             and folds every pruned row's candidates into its packed 64-bit
+//             running maximum, so the (V x k) similarity matrix never reaches HBM.
+//
+// One CTA computes a 128 x BN tile.  Warp 0 streams 128x64 / BNx64 operand tiles
+// with TMA into a ring of 128-byte-swizzled stages; one thread of warp 1 issues
+// tcgen05.mma (M = 128, N = BN, K = 16) into a TMEM accumulator; warps 2..5 read
+// the accumulator back with tcgen05.ld (one row per thread) and run the epilogue.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace {
+
+constexpr int kBM = 128, kBK = 64;
+constexpr int kGemmThreads = 192;
+
+enum { kEpiProj = 0, kEpiSim = 1 };
+
+struct GemmParams {
+  int num_k_blocks;           // K / 64
+  // projection
+  __nv_bfloat16* out[3];      // q, k, v
+  int out_rows;               // total tokens
+  int out_cols;               // D
+  // similarity
+  const int32_t* cu_seqlens; const int32_t* cu_vis; const int32_t* cu_kept; const int32_t* assign;
+  const float* inv_norm; const float* inv_norm_kept;
+  unsigned long long* best; float* sim_debug; int max_kept;
+  int* dev_status;
+};
+
+template <int BN> struct GemmSmem {
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2;
+  static constexpr int kBytes = kStages * (kABytes + kBBytes) + 1024 /*alignment slack*/ + 256 /*barriers*/ + BN * 4;
+};
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
+  using S = GemmSmem<BN>;
+  constexpr int kStages = S::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a_s = smem;
+  uint8_t* b_s = smem + kStages * S::kABytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * (S::kABytes + S::kBBytes));
+  uint64_t* empty = full + kStages;
+  uint64_t* acc_full = empty + kStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* ink_s = reinterpret_cast<float*>(smem + kStages * (S::kABytes + S::kBBytes) + 256);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN;
+
+  // tile coordinates in the operand matrices
+  int a_row = m0, b_row = n0;
+  int b = 0, Vb = 0, kb = 0, v0 = 0, k0 = 0;
+  if (EPI == kEpiSim) {
+    b = blockIdx.z;
+    v0 = p.cu_vis[b]; Vb = p.cu_vis[b + 1] - v0;
+    k0 = p.cu_kept[b]; kb = p.cu_kept[b + 1] - k0;
+    if (m0 >= Vb || n0 >= kb) return;          // uniform over the CTA, before any barrier or allocation
+    a_row = p.cu_seqlens[b] + m0;
+    b_row = k0 + n0;
+  }
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    ptx::mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 2) { ptx::tmem_alloc(tmem_slot, BN); ptx::tmem_relinquish(); }
+  if (EPI == kEpiSim) {
+    for (int j = threadIdx.x; j < BN; j += kGemmThreads) ink_s[j] = (n0 + j < kb) ? p.inv_norm_kept[k0 + n0 + j] : 0.f;
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tmap_a);
+      ptx::prefetch_tensormap(&tmap_b);
+      for (int kbk = 0; kbk < p.num_k_blocks; ++kbk) {
+        const int s = kbk % kStages;
+        if (!ptx::mbar_wait(&empty[s], ((kbk / kStages) & 1) ^ 1, abort_flag, p.dev_status)) break;
+        ptx::mbar_arrive_expect_tx(&full[s], S::kABytes + S::kBBytes);
+        ptx::tma_load_2d(a_s + s * S::kABytes, &tmap_a, &full[s], kbk * kBK, a_row);
+        ptx::tma_load_2d(b_s + s * S::kBBytes, &tmap_b, &full[s], kbk * kBK, b_row);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, BN, 0, 0);
+      bool ok = true;
+      for (int kbk = 0; kbk < p.num_k_blocks && ok; ++kbk) {
+        const int s = kbk % kStages;
+        ok = ptx::mbar_wait(&full[s], (kbk / kStages) & 1, abort_flag, p.dev_status);
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t a_addr = ptx::smem_u32(a_s + s * S::kABytes), b_addr = ptx::smem_u32(b_s + s * S::kBBytes);
+#pragma unroll
+        for (int kk = 0; kk < kBK / 16; ++kk) {
+          ptx::mma_ss(tmem_acc, ptx::smem_desc_kmajor_sw128(a_addr + kk * 32), ptx::smem_desc_kmajor_sw128(b_addr + kk * 32),
+                      idesc, (kbk > 0 || kk > 0) ? 1u : 0u);
+        }
+        ptx::mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+      }
+      if (ok) ptx::mma_commit(acc_full);
+    }
+  } else {
+    // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;           // row of the tile owned by this thread
+    const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full, 0, abort_flag, p.dev_status));
+    ptx::tc_fence_after_sync();
+    if (ok) {
+      const uint32_t t_row = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+      if (EPI == kEpiProj) {
+        const int grow = m0 + row;
+        const int which = n0 / p.out_cols, col0 = n0 % p.out_cols;   // BN divides D: a tile lies in one of q, k, v
+        __nv_bfloat16* dst = p.out[which] + (size_t)grow * p.out_cols + col0;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_row + c, r);
+          ptx::tmem_wait_ld();
+          if (grow < p.out_rows) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * j]), __uint_as_float(r[i + 2 * j + 1]));
+                w[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(dst + c + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else {
+        const int m = m0 + row;
+        const int g = v0 + m;
+        const bool active = m < Vb && p.assign[g] < 0;     // a pruned token of this request
+        const float inm = active ? p.inv_norm[g] : 0.f;
+        unsigned long long mine = 0ull;
+        float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + n0 : nullptr;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_row + c, r);
+          ptx::tmem_wait_ld();
+          if (active) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int sidx = n0 + c + i;
+              if (sidx < kb) {
+                const float sim = (__uint_as_float(r[i]) * inm) * ink_s[c + i];   // the value the arg-max compares
+                const unsigned long long packed =
+                    ((unsigned long long)ordered_key(sim) << 32) | (0xffffffffu - (unsigned)sidx);
+                mine = packed > mine ? packed : mine;
+                if (dbg != nullptr) dbg[c + i] = sim;
+              }
+            }
+          }
+        }
+        if (active) atomicMax(p.best + g, mine);
+      }
+    }
+    ptx::tc_fence_before_sync();
+  }
+  __syncthreads();
+  if (warp == 2) ptx::tmem_dealloc(tmem_acc, BN);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+template <int BN, int EPI>
+int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, dim3 grid, cudaStream_t s) {
+  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           GemmSmem<BN>::kBytes));
+  gemm_tc_kernel<BN, EPI><<<grid, kGemmThreads, GemmSmem<BN>::kBytes, s>>>(ta, tb, p);
+  D3TOM_LAUNCH_CHECK(ctx);
+  return D3TOM_OK;
+}
+
+}  // namespace
+
+int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
+                      uint32_t box_rows, uint32_t box_cols) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return -1;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_elems * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : (int)r;
+}
+
+int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int D, void* q, void* k, void* v,
+                   cudaStream_t s) {
+  constexpr int BN = 256;
+  if (D % BN != 0) {
+    // narrow models: fall back to 128-wide tiles (D % 64 == 0 is checked by the caller)
+    if (D % 128 != 0) return D3TOM_ERR_UNSUPPORTED;
+  }
+  CUtensorMap ta, tb;
+  int r = make_tmap_bf16_2d(&ta, x, (uint64_t)total, (uint64_t)D, (uint64_t)D, kBM);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  GemmParams p = {};
+  p.num_k_blocks = D / kBK;
+  p.out[0] = static_cast<__nv_bfloat16*>(q); p.out[1] = static_cast<__nv_bfloat16*>(k); p.out[2] = static_cast<__nv_bfloat16*>(v);
+  p.out_rows = total; p.out_cols = D; p.dev_status = ctx->dev_status;
+  if (D % BN == 0) {
+    r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, BN);
+    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+    return launch_gemm<256, kEpiProj>(ctx, ta, tb, p, dim3(ceil_div(total, kBM), 3 * D / 256, 1), s);
+  }
+  r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 128);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  return launch_gemm<128, kEpiProj>(ctx, ta, tb, p, dim3(ceil_div(total, kBM), 3 * D / 128, 1), s);
+}
+
+int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
+  if (a.D % kBK != 0) return D3TOM_ERR_UNSUPPORTED;
+  CUtensorMap ta, tb;
+  int r = make_tmap_bf16_2d(&ta, a.hidden, (uint64_t)a.total_tokens, (uint64_t)a.D, (uint64_t)a.D, kBM);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  const int kept_rows_bound = a.total_tokens;    // rows the kept-row scratch can hold
+  r = make_tmap_bf16_2d(&tb, ctx->kept_rows, (uint64_t)kept_rows_bound, (uint64_t)a.D, (uint64_t)a.D, 128);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  GemmParams p = {};
+  p.num_k_blocks = a.D / kBK;
+  p.cu_seqlens = a.cu_seqlens; p.cu_vis = a.cu_vis; p.cu_kept = a.cu_kept; p.assign = a.assign;
+  p.inv_norm = ctx->inv_norm; p.inv_norm_kept = ctx->inv_norm_kept; p.best = ctx->best; p.sim_debug = a.sim_debug;
+  p.max_kept = a.max_kept; p.dev_status = ctx->dev_status;
+  return launch_gemm<128, kEpiSim>(ctx, ta, tb, p, dim3(ceil_div(a.max_visual, kBM), ceil_div(a.max_kept, 128), a.B), s);
+}

@@ -1,0 +1,123 @@
+"""One merge-layer step as a chain of C-ABI calls on one stream:
+
+    d3tom_attn_importance -> d3tom_select -> d3tom_merge
+        -> n_post x (d3tom_proj_qkv -> d3tom_attn_varlen)
+
+This class only owns device buffers and marshals sizes; every step of the path
+runs inside the library's kernels.  Sizes that the C ABI takes from the host
+(keep counts, prefix sums of kept counts and of the shortened lengths) are
+computed here from the request shapes; nothing is read back from the device
+between the calls.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B_
+
+
+def _i32(a, device):
+    return torch.as_tensor(np.asarray(a, dtype=np.int32), device=device)
+
+
+class MergeLayerStep:
+    def __init__(self, H: int, dh: int, dtype: torch.dtype, max_total_tokens: int, max_batch: int,
+                 max_deciders: int, max_visual_per_request: int, n_post: int = 0, mode: int = B_.AGG_MEAN,
+                 sim_debug: bool = False, device: int = 0):
+        self.H, self.dh, self.D = H, dh, H * dh
+        self.dtype = dtype
+        self.dev = torch.device("cuda", device)
+        self.mode = mode
+        self.n_post = n_post
+        self.want_sim_debug = sim_debug
+        self.ctx = B_.Context(max_total_tokens, max_batch, H, dh, max(1, max_deciders), max_visual_per_request, device)
+        T = max_total_tokens
+        kw = dict(device=self.dev)
+        self.attn_out = torch.empty(T, self.D, dtype=dtype, **kw)
+        self.importance = torch.empty(T, dtype=torch.float32, **kw)
+        self.kept_idx = torch.empty(T, dtype=torch.int32, **kw)
+        self.keep_mask = torch.empty(T, dtype=torch.uint8, **kw)
+        self.assign = torch.empty(T, dtype=torch.int32, **kw)
+        self.member_count = torch.empty(T, dtype=torch.int32, **kw)
+        self.src_of_dst = torch.empty(T, dtype=torch.int32, **kw)
+        self.hidden_out = torch.empty(T, self.D, dtype=dtype, **kw)
+        self.sim_debug = None
+        if n_post:
+            self.q2 = torch.empty(T, self.D, dtype=dtype, **kw)
+            self.k2 = torch.empty(T, self.D, dtype=dtype, **kw)
+            self.v2 = torch.empty(T, self.D, dtype=dtype, **kw)
+            self.layer_out = [torch.empty(T, self.D, dtype=dtype, **kw) for _ in range(n_post)]
+        self.scale = 1.0 / float(np.sqrt(dh))
+
+    # ------------------------------------------------------------------ problem description (small index arrays)
+    def set_problem(self, n_visual: Sequence[int], n_prompt: Sequence[int], n_resp: Sequence[int],
+                    decider_pos: List[np.ndarray], keep_count: Sequence[int]):
+        """Uploads the index arrays of a batch.  keep_count[b] = number of kept
+        visual tokens of request b (from d3tom_keep_count); a request without
+        deciders must be given keep_count = n_visual (Algorithm 1, else-branch)."""
+        self.nB = len(n_visual)
+        self.n_visual_h = [int(x) for x in n_visual]
+        self.seqlens_h = [int(v + p + o) for v, p, o in zip(n_visual, n_prompt, n_resp)]
+        self.keep_h = [int(x) for x in keep_count]
+        self.out_lens_h = [n - v + k for n, v, k in zip(self.seqlens_h, self.n_visual_h, self.keep_h)]
+        cs = lambda a: np.concatenate([[0], np.cumsum(a)]).astype(np.int32)
+        self.cu_seqlens_h, self.cu_vis_h = cs(self.seqlens_h), cs(self.n_visual_h)
+        self.cu_kept_h, self.cu_out_h = cs(self.keep_h), cs(self.out_lens_h)
+        self.cu_dec_h = cs([len(d) for d in decider_pos])
+        dec = np.concatenate([np.asarray(d, dtype=np.int32) for d in decider_pos]) if self.cu_dec_h[-1] else np.zeros(1, np.int32)
+        d = self.dev
+        self.cu_seqlens, self.cu_vis = _i32(self.cu_seqlens_h, d), _i32(self.cu_vis_h, d)
+        self.cu_kept, self.cu_out = _i32(self.cu_kept_h, d), _i32(self.cu_out_h, d)
+        self.cu_dec, self.dec_pos = _i32(self.cu_dec_h, d), _i32(dec, d)
+        self.n_visual_d, self.keep_d = _i32(self.n_visual_h, d), _i32(self.keep_h, d)
+        self.total = int(self.cu_seqlens_h[-1])
+        self.total_vis = int(self.cu_vis_h[-1])
+        self.total_kept = int(self.cu_kept_h[-1])
+        self.total_out = int(self.cu_out_h[-1])
+        self.max_seqlen, self.max_visual = max(self.seqlens_h), max(self.n_visual_h)
+        self.max_kept, self.max_out = max(self.keep_h), max(self.out_lens_h)
+        if self.want_sim_debug:
+            self.sim_debug = torch.full((self.total_vis, self.max_kept), float("nan"), dtype=torch.float32, device=d)
+
+    # ------------------------------------------------------------------ the calls
+    def attn_importance(self, q, k, v, stream=None):
+        self.ctx.d3tom_attn_importance(q, k, v, self.cu_seqlens, self.n_visual_d, self.dec_pos, self.cu_dec, self.nB,
+                                       self.total, self.max_seqlen, self.max_visual, int(self.cu_dec_h[-1]),
+                                       self.scale, self.attn_out, self.importance, self.cu_vis, stream)
+
+    def select(self, stream=None):
+        self.ctx.d3tom_select(self.importance, self.cu_vis, self.keep_d, self.cu_kept, self.nB, self.max_visual,
+                              self.kept_idx, self.keep_mask, stream)
+
+    def merge(self, hidden=None, stream=None):
+        hidden = self.attn_out if hidden is None else hidden
+        self.ctx.d3tom_merge(self.mode, hidden, self.cu_seqlens, self.n_visual_d, self.cu_vis, self.kept_idx,
+                             self.cu_kept, self.nB, self.D, self.total, self.total_out, self.max_visual,
+                             self.max_kept, self.hidden_out, self.cu_out, self.assign, self.member_count,
+                             self.src_of_dst, self.sim_debug, stream)
+
+    def post_layer(self, l: int, x, w_qkv, stream=None):
+        self.ctx.d3tom_proj_qkv(x, w_qkv, self.total_out, self.D, self.q2, self.k2, self.v2, stream)
+        self.ctx.d3tom_attn_varlen(self.q2, self.k2, self.v2, self.cu_out, self.nB, self.total_out, self.max_out,
+                                   self.scale, self.layer_out[l], stream)
+
+    def run(self, q, k, v, w_post: Optional[Sequence[torch.Tensor]] = None, stream=None):
+        """Enqueue the whole step.  Returns the last tensor of the chain."""
+        self.attn_importance(q, k, v, stream)
+        self.select(stream)
+        self.merge(stream=stream)
+        x = self.hidden_out
+        for l in range(self.n_post):
+            self.post_layer(l, x, w_post[l], stream)
+            x = self.layer_out[l]
+        return x
+
+    def launches_per_step(self) -> int:
+        """Kernels of this library launched by one run(): attention 1 + importance finish 2,
+        select 1, merge 3 (prepare) + 1 (similarity, when something is pruned) + 2 (finish),
+        and 2 per post-merge layer."""
+        sim = 1 if self.total_out < self.total else 0
+        return 3 + 1 + 3 + sim + 2 + 2 * self.n_post

@@ -1,0 +1,180 @@
+"""Edge cases of the CUDA path against the oracle: ragged tails, several tiles,
+degenerate keep counts and decider sets, adversarial select inputs, host-made
+argument errors."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import d3tom_oracle as orc
+from paper_2511_12280_b200 import binding as B_
+from paper_2511_12280_b200 import workload as wl
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def small(dtype="bf16", H=2, dh=128, seed=11, reqs=None, post=1):
+    reqs = reqs or [dict(V=300, P=17, O=24, n_dec=5, r=0.3), dict(V=129, P=1, O=8, n_dec=1, r=0.1),
+                    dict(V=517, P=40, O=33, n_dec=33, r=0.5)]
+    return wl.make_workload("small", dtype, H, dh, seed, 16, reqs, post_layers=post)
+
+
+@pytest.mark.parametrize("dh", [128, 64])
+@pytest.mark.parametrize("mode", [B_.AGG_MEAN, B_.AGG_SUM])
+def test_ragged_batch_tensor_core_path(dh, mode):
+    pu.check_step(small(dh=dh, H=2 if dh == 128 else 3), mode=mode)
+
+
+def test_ragged_batch_fp32_path():
+    pu.check_step(small(dtype="fp32", dh=32, H=2, post=1))
+
+
+def test_lengths_around_tile_boundaries():
+    # one, two and three 128-row tiles with 1-row tails, exact multiples, and a tiny request
+    reqs = [dict(V=100, P=20, O=8, n_dec=2, r=0.25), dict(V=120, P=4, O=5, n_dec=5, r=0.25),
+            dict(V=240, P=8, O=8, n_dec=3, r=0.25), dict(V=250, P=3, O=4, n_dec=1, r=0.25),
+            dict(V=2, P=1, O=1, n_dec=1, r=0.5), dict(V=380, P=3, O=2, n_dec=2, r=0.25)]
+    pu.check_step(small(reqs=reqs, post=1))
+
+
+def test_keep_ratio_one_is_identity():
+    w = small(post=0)
+    step = pu.make_step(w, keep_count=list(w.n_visual), sim_debug=False)
+    dev = step.dev
+    q, k, v = w.q_for().to(dev), w.k.to(dev), w.v.to(dev)
+    step.run(q, k, v)
+    torch.cuda.synchronize()
+    total = step.total
+    assert step.total_out == total
+    assert torch.equal(step.hidden_out[:total], step.attn_out[:total])          # bit for bit
+    assert step.src_of_dst[:total].cpu().tolist() == list(range(total))
+    assert not step.member_count[:step.total_kept].any()
+    assert step.keep_mask[:step.total_vis].all()
+    step.ctx.close()
+
+
+def test_keep_one_token_everything_merges_into_it():
+    w = small(post=0)
+    pu.check_step(w, keep_count=[1, 1, 1])
+    pu.check_step(w, keep_count=[1, 1, 1], mode=B_.AGG_SUM)
+
+
+def test_no_deciders_gives_zero_importance_and_identity():
+    w = small(post=0)
+    dec = [np.zeros(0, np.int32) for _ in range(w.B)]
+    pu.check_step(w, decider_pos=dec)                      # keep_count defaults to |V| without deciders
+
+
+def test_mixed_decider_counts_and_single_decider():
+    w = small(post=0)
+    dec = [w.decider_pos[0][:1], np.zeros(0, np.int32), w.decider_pos[2]]
+    pu.check_step(w, decider_pos=dec)
+
+
+def test_duplicate_rows_and_heavy_slots():
+    # many identical visual rows: cosine ties resolve to the lowest kept position and
+    # some kept tokens collect far more than 32 members (the long-list aggregation path)
+    w = small(post=0, reqs=[dict(V=400, P=8, O=8, n_dec=4, r=0.02)])
+    w.k[:400] = w.k[:1]
+    w.v[5:400] = w.v[5:6]
+    pu.check_step(w)
+    pu.check_step(w, mode=B_.AGG_SUM)
+
+
+def run_select(scores_list, ks):
+    B = len(scores_list)
+    V = [len(s) for s in scores_list]
+    cu_vis = np.concatenate([[0], np.cumsum(V)]).astype(np.int32)
+    cu_kept = np.concatenate([[0], np.cumsum(ks)]).astype(np.int32)
+    ctx = B_.Context(max(8, int(cu_vis[-1])), B, 1, 64, 1, max(V))
+    dev = torch.device("cuda", 0)
+    imp = torch.as_tensor(np.concatenate(scores_list).astype(np.float32), device=dev)
+    t = lambda a: torch.as_tensor(np.asarray(a, np.int32), device=dev)
+    kept = torch.full((int(cu_kept[-1]),), -7, dtype=torch.int32, device=dev)
+    mask = torch.full((int(cu_vis[-1]),), 9, dtype=torch.uint8, device=dev)
+    ctx.d3tom_select(imp, t(cu_vis), t(ks), t(cu_kept), B, max(V), kept, mask)
+    torch.cuda.synchronize()
+    kept, mask = kept.cpu().numpy(), mask.cpu().numpy()
+    for b in range(B):
+        want = orc.select(scores_list[b].astype(np.float32), ks[b])
+        assert np.array_equal(kept[cu_kept[b]:cu_kept[b + 1]], want), b
+        m = np.zeros(V[b], np.uint8); m[want] = 1
+        assert np.array_equal(mask[cu_vis[b]:cu_vis[b + 1]], m), b
+    ctx.close()
+
+
+def test_select_adversarial_inputs():
+    rng = np.random.default_rng(5)
+    run_select([np.full(1000, 0.25), np.full(33, 0.0), np.full(1, 3.0)], [400, 33, 1])      # all equal
+    run_select([rng.integers(0, 4, 5000) / 8.0, rng.integers(0, 2, 1025) * 1.0], [1234, 1])  # few distinct values
+    run_select([rng.random(4096), rng.random(777) * 1e-30, rng.random(2048) * 1e30], [1024, 700, 2048])
+    x = rng.random(3000).astype(np.float32)
+    x[1000:2000] = x[1500]                               # a long run of ties straddling the threshold
+    run_select([x], [int((x > x[1500]).sum()) + 37])
+    # keys that differ only in the lowest mantissa bits
+    base = np.float32(0.37)
+    y = np.array([np.nextafter(base, np.float32(1), dtype=np.float32) if i % 3 == 0 else base for i in range(2000)], np.float32)
+    run_select([y], [700])
+    run_select([rng.random(70000)], [12345])             # larger than the shared-memory staging
+
+
+def test_host_made_failures_return_status_codes():
+    w = small(post=0)
+    step = pu.make_step(w, sim_debug=False)
+    dev = step.dev
+    q, k, v = w.q_for().to(dev), w.k.to(dev), w.v.to(dev)
+    lib = B_.load()
+    h = step.ctx._h
+    s = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    P = lambda t: ctypes.c_void_p(t.data_ptr())
+    # workspace limits
+    assert lib.d3tom_attn_varlen(h, B_.BF16, P(q), P(k), P(v), P(step.cu_seqlens), step.nB, step.total + 1,
+                                 step.max_seqlen, 0.1, P(step.attn_out), s) == B_.ERR_WORKSPACE
+    assert lib.d3tom_attn_varlen(h, B_.BF16, P(q), P(k), P(v), P(step.cu_seqlens), step.nB + 1, step.total,
+                                 step.max_seqlen, 0.1, P(step.attn_out), s) == B_.ERR_WORKSPACE
+    # invalid arguments
+    assert lib.d3tom_attn_varlen(h, B_.BF16, None, P(k), P(v), P(step.cu_seqlens), step.nB, step.total,
+                                 step.max_seqlen, 0.1, P(step.attn_out), s) == B_.ERR_INVALID_ARG
+    assert lib.d3tom_attn_varlen(h, B_.BF16, P(q), P(k), P(v), P(step.cu_seqlens), step.nB, step.total,
+                                 step.max_seqlen, -1.0, P(step.attn_out), s) == B_.ERR_INVALID_ARG
+    assert lib.d3tom_attn_varlen(h, 7, P(q), P(k), P(v), P(step.cu_seqlens), step.nB, step.total,
+                                 step.max_seqlen, 0.1, P(step.attn_out), s) == B_.ERR_UNSUPPORTED
+    with pytest.raises(B_.D3tomError) as e:
+        step.ctx.d3tom_merge(5, step.attn_out, step.cu_seqlens, step.n_visual_d, step.cu_vis, step.kept_idx,
+                             step.cu_kept, step.nB, step.D, step.total, step.total_out, step.max_visual,
+                             step.max_kept, step.hidden_out, step.cu_out, step.assign, step.member_count,
+                             step.src_of_dst)
+    assert e.value.status == B_.ERR_INVALID_ARG
+    # unsupported head_dim for the tensor-core path
+    with pytest.raises(B_.D3tomError) as e:
+        bad = B_.Context(256, 1, 2, 96, 1, 128)
+        x = torch.zeros(256, 2, 96, dtype=torch.bfloat16, device=dev)
+        bad.d3tom_attn_varlen(x, x, x, step.cu_seqlens, 1, 256, 256, 0.1, x)
+    assert e.value.status == B_.ERR_UNSUPPORTED
+    # the context is still usable afterwards
+    step.run(q, k, v)
+    torch.cuda.synchronize()
+    assert step.ctx.device_status() == 0
+    step.ctx.close()
+
+
+def test_results_are_reproducible_run_to_run():
+    w = small(post=1)
+    step = pu.make_step(w, sim_debug=False)
+    dev = step.dev
+    q, k, v = w.q_for().to(dev), w.k.to(dev), w.v.to(dev)
+    wp = [x.to(dev) for x in w.w_post]
+    outs = []
+    for _ in range(3):
+        y = step.run(q, k, v, wp)
+        torch.cuda.synchronize()
+        outs.append((step.importance[:step.total_vis].clone(), step.kept_idx[:step.total_kept].clone(),
+                     step.assign[:step.total_vis].clone(), step.hidden_out[:step.total_out].clone(),
+                     y[:step.total_out].clone()))
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+    step.ctx.close()
