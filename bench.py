@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the D3ToM merge-layer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch of synthetic input:
+merge-layer attention + importance map, select, merge (similarity, aggregation,
+compaction) and the post-merge layers (projection + ragged attention each).
+The default workload is C2, the LLaDA-8B-shaped configuration with thousands of
+visual tokens (4096 visual + 128 prompt + 64 response tokens, keep ratio 0.25,
+3 post-merge layers).  One JSON line is printed by rank 0.
+
+With N > 1 (launched by torch.distributed.run) every rank processes its own
+request of the same shape: the path shards by request, with no collective on
+the data path; the only communication is the barrier and the max-over-ranks of
+the timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOAD_TEXT = {
+    "C0": "C0: tiny fp32 merge layer, 256 visual + 16 prompt + 16 response tokens, 4 heads x 64, keep 0.25",
+    "C1": "C1: LLaDA-8B-shaped merge layer, 1024 visual + 64 prompt + 64 response tokens, 32 heads x 128, keep 0.10",
+    "C2": "C2: LLaDA-8B-shaped, 4096 visual + 128 prompt + 64 response tokens, 32 heads x 128, keep 0.25, 3 post-merge layers",
+    "C4": "C4: 8 ragged requests, 1024-4096 visual tokens each, 32 heads x 128, keep in {0.1,0.25,0.5}, 3 post-merge layers",
+}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.idx = device_index
+        self.proc = None
+        self.path = None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.path is None:
+            return out
+        try:
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.strip().lower() == "active":
+                    reasons.add(name)
+        if sm:
+            # the median over the busiest half: the sampler also sees the idle edges of the region
+            top = sorted(sm)[len(sm) // 2:]
+            out.update(sm_mhz=float(np.median(top)), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------ oracle timing
+def oracle_step_sample(w, heads=2, row_frac=8):
+    """Times the CPU oracle, as it stands, on a bounded sample of one step of
+    workload ``w`` and extrapolates linearly to the full step:
+    attention and importance on ``heads`` of the H heads (x H/heads), select and
+    merge in full, one post-merge layer with its projection on 1/row_frac of the
+    rows (x row_frac) and its attention on ``heads`` heads (x H/heads), times the
+    number of post-merge layers.  Returns (seconds per full step, description)."""
+    from oracle import d3tom_oracle as orc
+    H, dh = w.H, w.dh
+    hs = min(heads, H)
+    scale = 1.0 / np.sqrt(dh)
+    cu = w.cu_seqlens
+    q = w.q_for().to(dtype=__import__("torch").float64).numpy()
+    k = w.k.double().numpy()
+    v = w.v.double().numpy()
+    dec = np.concatenate([np.asarray(d, np.int64) for d in w.decider_pos])
+    t = {}
+    t0 = time.perf_counter()
+    out_h = orc.attention(q[:, :hs], k[:, :hs], v[:, :hs], cu, scale)
+    t["attn"] = (time.perf_counter() - t0) * H / hs
+    t0 = time.perf_counter()
+    S = orc.importance(q[:, :hs], k[:, :hs], cu, w.n_visual, dec, w.cu_deciders(), scale)
+    t["importance"] = (time.perf_counter() - t0) * H / hs
+    t0 = time.perf_counter()
+    kept = [orc.select(S[b].astype(np.float32), orc.keep_count(w.n_visual[b], w.keep_ratio[b])) for b in range(w.B)]
+    t["select"] = time.perf_counter() - t0
+    hidden = np.zeros((q.shape[0], H * dh))
+    hidden[:, :hs * dh] = out_h
+    hidden = orc.round_storage(hidden, w.dtype)
+    t0 = time.perf_counter()
+    res = orc.merge(hidden, cu, w.n_visual, kept, orc.MEAN, w.dtype)
+    t["merge"] = time.perf_counter() - t0
+    t["post"] = 0.0
+    if w.w_post:
+        x = res["hidden_out"]
+        wq = w.w_post[0].double().numpy()
+        n_sub = max(1, x.shape[0] // row_frac)
+        t0 = time.perf_counter()
+        orc.proj_qkv(x[:n_sub], wq, H, w.dtype)
+        t_proj = (time.perf_counter() - t0) * x.shape[0] / n_sub
+        qq = x.reshape(x.shape[0], H, dh)[:, :hs]
+        t0 = time.perf_counter()
+        orc.attention(qq, qq, qq, res["cu_seqlens_out"], scale)
+        t_att = (time.perf_counter() - t0) * H / hs
+        t["post"] = (t_proj + t_att) * len(w.w_post)
+    desc = ("oracle on %d of %d heads for attention/importance (x%d), select+merge in full, one post-merge layer "
+            "(projection on 1/%d of the rows, attention on %d heads) x%d layers; extrapolated linearly"
+            % (hs, H, H // hs, row_frac, hs, len(w.w_post)))
+    return sum(t.values()), desc, t
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="C2", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2511_12280_b200 import workload as wl
+    config = {"workload": WORKLOAD_TEXT[args.config], "requests_per_gpu": None, "aggregation": "mean",
+              "l2": "inputs larger than L2 (per-step working set > 126 MB)", "parallelism": "request-sharded replicas x%d" % world}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        w = wl.config(args.config)
+        config["requests_per_gpu"] = w.B
+        times = []
+        desc, parts = "", {}
+        for i in range(args.warmup + args.steps):
+            sec, desc, parts = oracle_step_sample(w)
+            if i >= args.warmup:
+                times.append(sec)
+        us = float(np.mean(times)) * 1e6
+        line = {"impl": "reference", "metric": "merge_layer_step_us", "value": us, "unit": "us", "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": us, "unit": "us", "cores": blas_threads(), "kind": "oracle", "sample": desc},
+                "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "breakdown_s": parts}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    import torch.distributed as dist
+    from paper_2511_12280_b200 import binding as B_
+    from paper_2511_12280_b200.pipeline import MergeLayerStep
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the merge-layer path has no CPU fallback")
+    B_.load()           # fails loudly if the CUDA library has not been built
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = wl.config(args.config)
+    config["requests_per_gpu"] = w.B
+    keep = [B_.d3tom_keep_count(v, r) for v, r in zip(w.n_visual, w.keep_ratio)]
+    total = int(w.cu_seqlens[-1])
+    step = MergeLayerStep(w.H, w.dh, w.torch_dtype, total, w.B, sum(len(d) for d in w.decider_pos), max(w.n_visual),
+                          n_post=len(w.w_post), mode=B_.AGG_MEAN, device=local_rank)
+    step.set_problem(w.n_visual, w.n_prompt, w.n_resp, w.decider_pos, keep)
+    q_h, k_h, v_h = (t.contiguous().pin_memory() for t in (w.q_for(), w.k, w.v))
+    q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
+    w_post = [x.to(dev) for x in w.w_post]
+    out_h = torch.empty(step.total_out, step.D, dtype=w.torch_dtype).pin_memory()
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) / iters * 1e3   # us
+
+    def max_over_ranks(x):
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing of the whole step
+    run = lambda: step.run(q, k, v, w_post)
+    for _ in range(max(3, args.warmup)):
+        run()
+    sync_all()
+    with ClockSampler(local_rank) as clk:
+        step_us = timed(run, args.steps)
+        sync_all()
+        # ---- per-call breakdown (each call timed back to back on warm instruction caches;
+        #      every call's working set is streamed from HBM or L2 as it would be inside the step)
+        reps = max(10, args.steps)
+        br = {}
+        br["attn_importance"] = timed(lambda: step.attn_importance(q, k, v), reps)
+        br["select"] = timed(lambda: step.select(), reps)
+        br["merge"] = timed(lambda: step.merge(), reps)
+        if step.n_post:
+            br["proj_qkv"] = timed(lambda: step.ctx.d3tom_proj_qkv(step.hidden_out, w_post[0], step.total_out, step.D,
+                                                                     step.q2, step.k2, step.v2), reps)
+            br["attn_varlen"] = timed(lambda: step.ctx.d3tom_attn_varlen(step.q2, step.k2, step.v2, step.cu_out, step.nB,
+                                                                        step.total_out, step.max_out, step.scale,
+                                                                        step.layer_out[0]), reps)
+        # the dominant kernel alone (no importance side-work): the attention kernel at the merge-layer length
+        attn_kernel_us = timed(lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
+                                                                  step.max_seqlen, step.scale, step.attn_out), reps)
+        sync_all()
+    clocks = clk.summary()
+    assert step.ctx.device_status() == 0, "device status word reports a kernel-side problem"
+
+    # ---- end to end through the C ABI with host buffers: H2D of Q,K,V, the step, D2H of the result
+    def e2e():
+        q.copy_(q_h, non_blocking=True); k.copy_(k_h, non_blocking=True); v.copy_(v_h, non_blocking=True)
+        y = step.run(q, k, v, w_post)
+        out_h.copy_(y[:step.total_out], non_blocking=True)
+    for _ in range(3):
+        e2e()
+    sync_all()
+    e2e_us = timed(e2e, max(5, args.steps // 2))
+    sync_all()
+
+    step_us_max = max_over_ranks(step_us)
+    e2e_us_max = max_over_ranks(e2e_us)
+
+    # ---- roofline of the dominant kernel (merge-layer attention): 4 N^2 D flops per request
+    peaks, peak_kind = load_peaks()
+    attn_flops = sum(4.0 * n * n * step.D for n in step.seqlens_h)
+    achieved = attn_flops / (attn_kernel_us * 1e-6) / 1e12
+    roofline = {"bound": "tensor", "kernel": "attn_tc_kernel (merge-layer attention, timed alone)",
+                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_kind": peak_kind + " burst"}
+    merge_bytes = (step.total + step.total_out) * step.D * q.element_size()
+    sim_flops = sum(2.0 * (v_ - k_) * k_ * step.D for v_, k_ in zip(step.n_visual_h, step.keep_h))
+    post_attn_flops = sum(4.0 * n * n * step.D for n in step.out_lens_h)
+    derived = {
+        "attn_importance_tflops": attn_flops / (br["attn_importance"] * 1e-6) / 1e12,
+        "merge_call_gbs": merge_bytes / (br["merge"] * 1e-6) / 1e9,
+        "merge_call_frac_of_hbm_peak": merge_bytes / (br["merge"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
+        "similarity_gflop": sim_flops / 1e9,
+    }
+    if step.n_post:
+        derived["attn_varlen_tflops"] = post_attn_flops / (br["attn_varlen"] * 1e-6) / 1e12
+        derived["proj_qkv_tflops"] = 2.0 * step.total_out * step.D * 3 * step.D / (br["proj_qkv"] * 1e-6) / 1e12
+
+    line = {
+        "metric": "merge_layer_step_us", "value": step_us_max / world, "unit": "us", "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": step_us_max / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
+        "steps_per_s": world / (step_us_max * 1e-6),
+        "e2e": {"value": e2e_us_max / world, "unit": "us",
+                "h2d_bytes_per_step": int(3 * q_h.numel() * q_h.element_size()),
+                "d2h_bytes_per_step": int(out_h.numel() * out_h.element_size())},
+        "gpu_launches": step.launches_per_step() * args.steps,
+        "roofline": roofline, "breakdown_us": br, "derived": derived, "clocks": clocks,
+        "peaks": dict(peaks, kind=peak_kind),
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sec, desc, parts = oracle_step_sample(w)
+        line["cpu_baseline"] = {"value": sec * 1e6, "unit": "us", "cores": blas_threads(), "kind": "oracle",
+                                "sample": desc, "breakdown_s": parts}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -25,7 +25,7 @@ def small(dtype="bf16", H=2, dh=128, seed=11, reqs=None, post=1):
 @pytest.mark.parametrize("dh", [128, 64])
 @pytest.mark.parametrize("mode", [B_.AGG_MEAN, B_.AGG_SUM])
 def test_ragged_batch_tensor_core_path(dh, mode):
-    pu.check_step(small(dh=dh, H=2 if dh == 128 else 3), mode=mode)
+    pu.check_step(small(dh=dh, H=2 if dh == 128 else 4), mode=mode)
 
 
 def test_ragged_batch_fp32_path():
