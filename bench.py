@@ -65,7 +65,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -78,6 +78,18 @@ class ClockSampler:
                 self.proc.wait(timeout=5)
             except Exception:
                 self.proc.kill()
+
+    def wait_started(self, keep_busy, limit_s=4.0):
+        """Runs ``keep_busy`` until the sampler has written its first line (nvidia-smi takes a
+        moment to start), so that the samples cover the timed region that follows."""
+        t0 = time.time()
+        while self.proc is not None and time.time() - t0 < limit_s:
+            keep_busy()
+            try:
+                if os.path.getsize(self.path) > 0:
+                    break
+            except OSError:
+                break
 
     def summary(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
@@ -172,11 +184,13 @@ def blas_threads():
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="C2", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "step"],
+                    help="profiling aid: after one full step, run just this call --steps times and exit")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -253,17 +267,37 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    # ---- device-resident timing of the whole step
     run = lambda: step.run(q, k, v, w_post)
+    if args.only is not None:
+        run()
+        calls = {
+            "attn_importance": lambda: step.attn_importance(q, k, v),
+            "select": lambda: step.select(),
+            "merge": lambda: step.merge(),
+            "proj_qkv": lambda: step.ctx.d3tom_proj_qkv(step.hidden_out, w_post[0], step.total_out, step.D,
+                                                        step.q2, step.k2, step.v2),
+            "attn_varlen": lambda: step.ctx.d3tom_attn_varlen(step.q2, step.k2, step.v2, step.cu_out, step.nB,
+                                                              step.total_out, step.max_out, step.scale,
+                                                              step.layer_out[0]),
+            "step": run,
+        }
+        torch.cuda.synchronize()
+        us = timed(calls[args.only], args.steps)
+        print(json.dumps({"only": args.only, "us": us, "config": args.config}))
+        return 0
+
+    # ---- device-resident timing of the whole step
     for _ in range(max(3, args.warmup)):
         run()
     sync_all()
     with ClockSampler(local_rank) as clk:
+        clk.wait_started(run)          # keeps the GPU busy until the sampler delivers
+        sync_all()
         step_us = timed(run, args.steps)
         sync_all()
         # ---- per-call breakdown (each call timed back to back on warm instruction caches;
         #      every call's working set is streamed from HBM or L2 as it would be inside the step)
-        reps = max(10, args.steps)
+        reps = min(100, max(10, args.steps))
         br = {}
         br["attn_importance"] = timed(lambda: step.attn_importance(q, k, v), reps)
         br["select"] = timed(lambda: step.select(), reps)
@@ -289,7 +323,7 @@ def main():
     for _ in range(3):
         e2e()
     sync_all()
-    e2e_us = timed(e2e, max(5, args.steps // 2))
+    e2e_us = timed(e2e, min(50, max(5, args.steps // 2)))
     sync_all()
 
     step_us_max = max_over_ranks(step_us)

@@ -187,27 +187,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[i], j & 1, abort_flag, a.dev_status));
         if (!ok) break;
         ptx::tc_fence_after_sync();
-        const int n_valid = min(kTile, n - j * kTile);       // keys of this tile that belong to the request
-        // ---- pass 1: row maximum (and the decider rows' raw scores)
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTile; c0 += 32) {
-          uint32_t r[32];
-          ptx::tmem_ld32(t_s + c0, r);
-          ptx::tmem_wait_ld();
-          if (c0 + 32 <= n_valid) {
+        // ---- the whole score row of this tile: 128 fp32 values, one TMEM lane
+        uint32_t sr[kTile];
+        ptx::tmem_ld32(t_s, sr);
+        ptx::tmem_ld32(t_s + 32, sr + 32);
+        ptx::tmem_ld32(t_s + 64, sr + 64);
+        ptx::tmem_ld32(t_s + 96, sr + 96);
+        ptx::tmem_wait_ld();
+        const int n_valid = n - j * kTile;                  // keys of this tile that belong to the request
+        if (n_valid < kTile) {                              // ragged last tile: keys past the end score -inf
 #pragma unroll
-            for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
-          } else {
+          for (int e = 0; e < kTile; ++e) if (e >= n_valid) sr[e] = 0xff800000u;
+        }
+        if (score_row != nullptr) {                         // decider row: raw scores over the visual keys
+          const int key0 = j * kTile;
 #pragma unroll
-            for (int e = 0; e < 32; ++e) if (c0 + e < n_valid) mx = fmaxf(mx, __uint_as_float(r[e]));
-          }
-          if (score_row != nullptr) {
-            const int key0 = j * kTile + c0;
+          for (int e = 0; e < kTile; e += 4) {
+            if (key0 + e + 3 < n_vis) {
+              *reinterpret_cast<float4*>(score_row + key0 + e) =
+                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
+                              __uint_as_float(sr[e + 3]));
+            } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) if (key0 + e < n_vis) score_row[key0 + e] = __uint_as_float(r[e]);
+              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
+            }
           }
         }
+        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
+              mx3 = __uint_as_float(sr[3]);
+#pragma unroll
+        for (int e = 4; e < kTile; e += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(sr[e]));     mx1 = fmaxf(mx1, __uint_as_float(sr[e + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(sr[e + 2])); mx3 = fmaxf(mx3, __uint_as_float(sr[e + 3]));
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         const float m_new = fmaxf(m_used, mx * c);
         const bool need = (m_new - m_used) > kRescaleThreshold;   // first tile: inf > threshold
         if (__any_sync(0xffffffffu, need)) {
@@ -227,38 +240,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           l_sum *= alpha;
           if (need) m_used = m_new;
         }
-        // ---- pass 2: p = exp2(s*c - m), row sum, bf16 P tile into the first 64 columns of S
-        // (64 keys at a time: both source chunks are read before the P chunk that overlaps them is written)
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTile; c0 += 64) {
-          uint32_t r0[32], r1[32], pk[32];
-          ptx::tmem_ld32(t_s + c0, r0);
-          ptx::tmem_ld32(t_s + c0 + 32, r1);
-          ptx::tmem_wait_ld();
-          float part = 0.f;
+        // ---- p = exp2(s*c - m), row sum, bf16 P tile into the first 64 columns of the S tile
+        const float neg_m = -m_used;
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float p0 = exp2f(fmaf(__uint_as_float(r0[e]), c, -m_used));
-            float p1 = exp2f(fmaf(__uint_as_float(r0[e + 1]), c, -m_used));
-            if (c0 + e >= n_valid) p0 = 0.f;
-            if (c0 + e + 1 >= n_valid) p1 = 0.f;
-            part += p0 + p1;
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-            pk[e >> 1] = *reinterpret_cast<uint32_t*>(&h2);
-          }
+        for (int half = 0; half < 2; ++half) {
+          uint32_t pk[32];
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float p0 = exp2f(fmaf(__uint_as_float(r1[e]), c, -m_used));
-            float p1 = exp2f(fmaf(__uint_as_float(r1[e + 1]), c, -m_used));
-            if (c0 + 32 + e >= n_valid) p0 = 0.f;
-            if (c0 + 32 + e + 1 >= n_valid) p1 = 0.f;
-            part += p0 + p1;
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-            pk[16 + (e >> 1)] = *reinterpret_cast<uint32_t*>(&h2);
+          for (int e = 0; e < 64; e += 4) {
+            const int x = half * 64 + e;
+            const float p0 = ptx::ex2(fmaf(__uint_as_float(sr[x]), c, neg_m));
+            const float p1 = ptx::ex2(fmaf(__uint_as_float(sr[x + 1]), c, neg_m));
+            const float p2 = ptx::ex2(fmaf(__uint_as_float(sr[x + 2]), c, neg_m));
+            const float p3 = ptx::ex2(fmaf(__uint_as_float(sr[x + 3]), c, neg_m));
+            sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+            __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
+            pk[e >> 1] = *reinterpret_cast<uint32_t*>(&h01);
+            pk[(e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h23);
           }
-          l_sum += part;
-          ptx::tmem_st32(t_s + (c0 >> 1), pk);             // keys c0..c0+63 -> P columns c0/2 .. c0/2+31
+          ptx::tmem_st32(t_s + half * 32, pk);             // keys 64*half .. +63 -> P columns 32*half .. +31
         }
+        l_sum += (sum0 + sum1) + (sum2 + sum3);
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
         ptx::mbar_arrive(&p_full[i]);
