@@ -225,6 +225,7 @@ def main():
     import torch.distributed as dist
     from paper_2511_12280_b200 import binding as B_
     from paper_2511_12280_b200.pipeline import MergeLayerStep
+    from paper_2511_12280_b200 import replicas
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the merge-layer path has no CPU fallback")
@@ -261,11 +262,7 @@ def main():
         return e0.elapsed_time(e1) / iters * 1e3   # us
 
     def max_over_ranks(x):
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, dev)
 
     run = lambda: step.run(q, k, v, w_post)
     if args.only is not None:
