@@ -124,6 +124,47 @@ int d3tom_attn_importance(d3tom_ctx* ctx, d3tom_dtype dt,
                           void* attn_out, float* importance, const int32_t* cu_vis,
                           d3tom_stream stream);
 
+/* Allocation-free variant of d3tom_attn_importance.  The paper has no
+ * counterpart: this exists for hosts that must not allocate device memory
+ * (a process whose memory pool owns the whole device, a sandbox that registers
+ * every allocation up front, a latency-critical loop that must stay off the
+ * allocator's device-wide lock) and therefore cannot call d3tom_create.
+ *
+ * It needs no context.  The scratch that the context would own lives in a
+ * fixed array inside the library image: about 10.1 MiB that every GPU
+ * loading the library holds until the process exits.  That array bounds the
+ * problem size; a call beyond any of
+ *     heads * max(1, n_deciders_total)                       <= D3TOM_STATIC_MAX_LSE_PAIRS
+ *     heads * total_tokens                                   <= D3TOM_STATIC_MAX_PARTIAL_FLOATS
+ *     heads * max(1, n_deciders_total) * round_up(max_visual, 4) <= D3TOM_STATIC_MAX_SCORE_FLOATS
+ * returns D3TOM_ERR_WORKSPACE and launches nothing (e.g. 32 heads x 16
+ * deciders x 4096 visual tokens, 16384 packed tokens, fits exactly).
+ *
+ * heads, head_dim replace the context's limits; every other argument is as in
+ * d3tom_attn_importance, and the results are the same bit for bit.  The work
+ * runs on the CURRENT device, which must be the one `stream` and the buffers
+ * belong to.  device_status_out (device, nullable) receives the kernels'
+ * status word at the end of the call (0, or D3TOM_ERR_TIMEOUT if a bounded
+ * wait ran out); read it after the stream has been waited for.
+ *
+ * The first call on each device looks up the array's device address; make
+ * that first call outside of any stream capture.  No call allocates or frees.
+ * All calls on a device share the one array, and it keeps what the previous
+ * call left there (this function clears the only word that has to start at
+ * zero): two calls that overlap on the GPU race with each other, so keep all
+ * calls of a device on one stream or order them with events. */
+#define D3TOM_STATIC_MAX_LSE_PAIRS      (1 << 14)
+#define D3TOM_STATIC_MAX_PARTIAL_FLOATS (1 << 19)
+#define D3TOM_STATIC_MAX_SCORE_FLOATS   (1 << 21)
+int d3tom_attn_importance_static(d3tom_dtype dt, int heads, int head_dim,
+                                 const void* q, const void* k, const void* v,
+                                 const int32_t* cu_seqlens, const int32_t* n_visual,
+                                 const int32_t* decider_pos, const int32_t* cu_deciders,
+                                 int B, int total_tokens, int max_seqlen, int max_visual, int n_deciders_total,
+                                 float softmax_scale,
+                                 void* attn_out, float* importance, const int32_t* cu_vis,
+                                 int32_t* device_status_out, d3tom_stream stream);
+
 /* Sec. 3.2.1, the partition V_kept / V_merge; Algorithm 1, TopK.
  *
  * Per request: the keep_count[b] visual tokens of highest importance, ordered by

@@ -48,6 +48,8 @@ _SIGNATURES = {
     "d3tom_keep_count": (_I, [_I, C.c_double]),
     "d3tom_schedule_alpha": (_I, [_I, _I, C.c_double, C.c_double, _I, C.POINTER(C.c_double)]),
     "d3tom_attn_importance": (_I, [_P, _I, _P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _F, _P, _P, _P, _P]),
+    "d3tom_attn_importance_static": (_I, [_I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _F, _P, _P, _P, _P,
+                                          _P]),
     "d3tom_select": (_I, [_P, _P, _P, _P, _P, _I, _I, _P, _P, _P]),
     "d3tom_merge": (_I, [_P, _I, _I, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
     "d3tom_attn_varlen": (_I, [_P, _I, _P, _P, _P, _P, _I, _I, _I, _F, _P, _P]),
@@ -112,6 +114,20 @@ def d3tom_schedule_alpha(step: int, T: int, a_min: float, a_max: float, reversed
     out = C.c_double()
     _check(load().d3tom_schedule_alpha(step, T, a_min, a_max, int(reversed_), C.byref(out)), "d3tom_schedule_alpha")
     return out.value
+
+
+def d3tom_attn_importance_static(heads, head_dim, q, k, v, cu_seqlens, n_visual, decider_pos, cu_deciders, B,
+                                 total_tokens, max_seqlen, max_visual, n_deciders_total, softmax_scale, attn_out,
+                                 importance, cu_vis, device_status_out=None, stream=None):
+    """d3tom_attn_importance for callers that may not allocate device memory: no context, the
+    scratch is a fixed array inside the library (see include/d3tom.h for its size limits).
+    Runs on the current device; calls on one device must not overlap."""
+    _check(load().d3tom_attn_importance_static(_dt(q), heads, head_dim, _ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens),
+                                               _ptr(n_visual), _ptr(decider_pos), _ptr(cu_deciders), B, total_tokens,
+                                               max_seqlen, max_visual, n_deciders_total, softmax_scale,
+                                               _ptr(attn_out), _ptr(importance), _ptr(cu_vis),
+                                               _ptr(device_status_out), _stream(stream)),
+           "d3tom_attn_importance_static")
 
 
 class Context:
