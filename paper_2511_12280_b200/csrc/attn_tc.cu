@@ -12,19 +12,26 @@
 //   warps 4-7   softmax of query tile 1
 //   warp  8     TMA producer: Q tiles once, then K_j / V_j tiles through a ring
 //   warp  9     one thread issues every tcgen05.mma
+//   warps 10-11 idle (they complete the third warpgroup so that registers can be
+//               moved from it to the softmax warpgroups with setmaxnreg)
 // TMEM (512 columns): S0 | S1 (128 fp32 columns each; the bf16 P tile overwrites
 // the first 64 columns of its S tile) | O0 | O1 (head_dim fp32 columns each).
 // Per key tile j and query tile i:  S_i = Q_i K_j^T  ->  softmax warps read S_i,
-// write P_i  ->  O_i += P_i V_j.  The running maximum is only raised when the
-// new one exceeds it by more than 2^8 (the O tile is then rescaled in place by
-// its own softmax warps); sums and outputs are exact for any reference maximum.
+// write P_i in two halves  ->  O_i += P_i V_j, the first half of the keys while
+// the second half is still being exponentiated.  The running maximum is only
+// raised when the new one exceeds it by more than 2^8 (the O tile is then
+// rescaled in place by its own softmax warps); sums and outputs are exact for
+// any reference maximum.  CTAs are issued from the END of each request towards
+// its beginning: the response rows (where the decider rows live and spill their
+// scores) are at the end, and the CTAs with extra work should not run last.
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace {
 
 constexpr int kTile = 128;            // query rows per tile and keys per tile
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 384;
+constexpr int kSoftmaxRegs = 216, kOtherRegs = 64;   // 256 * 216 + 128 * 64 <= 384 * 168
 constexpr int kKvSlots = 4;
 constexpr float kRescaleThreshold = 8.0f;
 
@@ -32,6 +39,26 @@ template <int DH> struct AttnSmem {
   static constexpr int kTileBytes = kTile * DH * 2;
   static constexpr int kBytes = 2 * kTileBytes + kKvSlots * kTileBytes + 1024 + 256;
 };
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// 32 lanes x 16 columns: the 16-register form of tcgen05.st
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 
 template <int DH>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -43,7 +70,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   constexpr int kHalves = DH / 64;
   const int b = blockIdx.z, h = blockIdx.y;
   const int lo = a.cu_seqlens[b], n = a.cu_seqlens[b + 1] - lo;
-  const int q0 = blockIdx.x * 2 * kTile;
+  const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * 2 * kTile;   // last rows of the request first
   if (q0 >= n) return;                                  // uniform; nothing allocated yet
   const int n_qt = (n - q0 > kTile) ? 2 : 1;
   const int n_kv = (n + kTile - 1) / kTile;
@@ -57,9 +84,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   uint64_t* kv_full = bars + 2;                         // [4]
   uint64_t* kv_empty = bars + 6;                        // [4]
   uint64_t* s_full = bars + 10;                         // [2]
-  uint64_t* p_full = bars + 12;                         // [2]
-  uint64_t* o_final = bars + 14;                        // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* p_lo = bars + 12;                           // [2]  P columns of keys 0..63 written (and O consistent)
+  uint64_t* p_hi = bars + 14;                           // [2]  P columns of keys 64..127 written
+  uint64_t* o_final = bars + 16;                        // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -67,7 +95,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&q_full[i], 1); ptx::mbar_init(&s_full[i], 1);
-      ptx::mbar_init(&p_full[i], kTile); ptx::mbar_init(&o_final[i], 1);
+      ptx::mbar_init(&p_lo[i], 4); ptx::mbar_init(&p_hi[i], 4);      // one arrival per softmax warp
+      ptx::mbar_init(&o_final[i], 1);
     }
     for (int s = 0; s < kKvSlots; ++s) { ptx::mbar_init(&kv_full[s], 1); ptx::mbar_init(&kv_empty[s], 1); }
     *abort_flag = 0;
@@ -81,82 +110,97 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   auto col_s = [](int i) -> uint32_t { return (uint32_t)i * 128u; };          // S_i (and P_i) columns
   auto col_o = [](int i) -> uint32_t { return 256u + (uint32_t)i * 128u; };   // O_i columns
 
-  if (warp == 8) {
-    // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      ptx::prefetch_tensormap(&tmap_q); ptx::prefetch_tensormap(&tmap_k); ptx::prefetch_tensormap(&tmap_v);
-      for (int i = 0; i < n_qt; ++i) {
-        ptx::mbar_arrive_expect_tx(&q_full[i], kTileBytes);
-        for (int hf = 0; hf < kHalves; ++hf)
-          ptx::tma_load_2d(q_s + i * kTileBytes + hf * kHalfBytes, &tmap_q, &q_full[i], h * DH + hf * 64,
-                           lo + q0 + i * kTile);
-      }
-      for (int it = 0; it < 2 * n_kv; ++it) {             // it = 2j: K_j, it = 2j+1: V_j
-        const int slot = it % kKvSlots, j = it >> 1;
-        if (!ptx::mbar_wait(&kv_empty[slot], ((it / kKvSlots) & 1) ^ 1, abort_flag, a.dev_status)) break;
-        ptx::mbar_arrive_expect_tx(&kv_full[slot], kTileBytes);
-        const CUtensorMap* tm = (it & 1) ? &tmap_v : &tmap_k;
-        for (int hf = 0; hf < kHalves; ++hf)
-          ptx::tma_load_2d(kv_s + slot * kTileBytes + hf * kHalfBytes, tm, &kv_full[slot], h * DH + hf * 64,
-                           lo + j * kTile);
-      }
-    }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(kTile, kTile, 0, 0);   // S = Q K^T, both K-major
-      constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kTile, DH, 0, 1);      // O += P V, V is MN-major
-      auto issue_qk = [&](int i, int slot) {
-        const uint32_t qa = ptx::smem_u32(q_s + i * kTileBytes), ka = ptx::smem_u32(kv_s + slot * kTileBytes);
-#pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (kk / 4) * kHalfBytes + (kk % 4) * 32;
-          ptx::mma_ss(tmem + col_s(i), ptx::smem_desc_kmajor_sw128(qa + off), ptx::smem_desc_kmajor_sw128(ka + off),
-                      idesc_qk, kk > 0 ? 1u : 0u);
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
+    if (warp == 8) {
+      // ------------------------------------------------------------ TMA producer
+      if (lane == 0) {
+        ptx::prefetch_tensormap(&tmap_q); ptx::prefetch_tensormap(&tmap_k); ptx::prefetch_tensormap(&tmap_v);
+        for (int i = 0; i < n_qt; ++i) {
+          ptx::mbar_arrive_expect_tx(&q_full[i], kTileBytes);
+          for (int hf = 0; hf < kHalves; ++hf)
+            ptx::tma_load_2d(q_s + i * kTileBytes + hf * kHalfBytes, &tmap_q, &q_full[i], h * DH + hf * 64,
+                             lo + q0 + i * kTile);
         }
-      };
-      auto issue_pv = [&](int i, int slot, bool accumulate) {
-        const uint32_t va = ptx::smem_u32(kv_s + slot * kTileBytes);
-#pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk) {            // 16 keys per instruction
-          ptx::mma_ts(tmem + col_o(i), tmem + col_s(i) + kk * 8,
-                      ptx::smem_desc_mnmajor_sw128(va + kk * 2048, kHalfBytes), idesc_pv,
-                      (accumulate || kk > 0) ? 1u : 0u);
+        for (int it = 0; it < 2 * n_kv; ++it) {             // it = 2j: K_j, it = 2j+1: V_j
+          const int slot = it % kKvSlots, j = it >> 1;
+          if (!ptx::mbar_wait(&kv_empty[slot], ((it / kKvSlots) & 1) ^ 1, abort_flag, a.dev_status)) break;
+          ptx::mbar_arrive_expect_tx(&kv_full[slot], kTileBytes);
+          const CUtensorMap* tm = (it & 1) ? &tmap_v : &tmap_k;
+          for (int hf = 0; hf < kHalves; ++hf)
+            ptx::tma_load_2d(kv_s + slot * kTileBytes + hf * kHalfBytes, tm, &kv_full[slot], h * DH + hf * 64,
+                             lo + j * kTile);
         }
-      };
-      bool ok = true;
-      for (int i = 0; i < n_qt && ok; ++i) ok = ptx::mbar_wait(&q_full[i], 0, abort_flag, a.dev_status);
-      if (ok) ok = ptx::mbar_wait(&kv_full[0], 0, abort_flag, a.dev_status);     // K_0
-      if (ok) {
-        ptx::tc_fence_after_sync();
-        for (int i = 0; i < n_qt; ++i) { issue_qk(i, 0); ptx::mma_commit(&s_full[i]); }
-        ptx::mma_commit(&kv_empty[0]);
       }
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int itv = 2 * j + 1, itk = 2 * j + 2;
-        const int vslot = itv % kKvSlots, kslot = itk % kKvSlots;
-        const bool more = j + 1 < n_kv;
-        for (int i = 0; i < n_qt && ok; ++i) {
-          ok = ptx::mbar_wait(&p_full[i], j & 1, abort_flag, a.dev_status);        // P_j(i) written, O_i consistent
-          if (ok && i == 0) ok = ptx::mbar_wait(&kv_full[vslot], (itv / kKvSlots) & 1, abort_flag, a.dev_status);
-          if (!ok) break;
+    } else if (warp == 9) {
+      // ------------------------------------------------------------ MMA issuer
+      // tcgen05.mma issue blocks once about two instructions are queued, so whatever this thread
+      // does between two MMAs is idle time of the tensor pipe: descriptors are built once and
+      // only advanced by one 32-bit add per instruction.
+      if (lane == 0) {
+        constexpr uint32_t idesc_qk = ptx::idesc_bf16_f32(kTile, kTile, 0, 0);   // S = Q K^T, both K-major
+        constexpr uint32_t idesc_pv = ptx::idesc_bf16_f32(kTile, DH, 0, 1);      // O += P V, V is MN-major
+        const ptx::SmemDesc q_desc[2] = {ptx::smem_desc_kmajor_sw128(ptx::smem_u32(q_s)),
+                                         ptx::smem_desc_kmajor_sw128(ptx::smem_u32(q_s + kTileBytes))};
+        const ptx::SmemDesc k_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(kv_s));
+        const ptx::SmemDesc v_desc0 = ptx::smem_desc_mnmajor_sw128(ptx::smem_u32(kv_s), kHalfBytes);
+        auto issue_qk = [&](int i, int slot) {
+          const ptx::SmemDesc qd = q_desc[i], kd = ptx::smem_desc_advance(k_desc0, slot * kTileBytes);
+#pragma unroll
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint32_t off = (kk / 4) * kHalfBytes + (kk % 4) * 32;
+            ptx::mma_ss(tmem + col_s(i), ptx::smem_desc_advance(qd, off), ptx::smem_desc_advance(kd, off), idesc_qk,
+                        kk > 0 ? 1u : 0u);
+          }
+        };
+        // keys 64*half .. 64*half+63 of the tile: P columns 32*half .., V rows 64*half ..
+        auto issue_pv_half = [&](int i, int slot, int half, bool accumulate) {
+          const ptx::SmemDesc vd = ptx::smem_desc_advance(v_desc0, slot * kTileBytes + half * 4 * 2048);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4) {                       // 16 keys per instruction
+            ptx::mma_ts(tmem + col_o(i), tmem + col_s(i) + (half * 4 + k4) * 8, ptx::smem_desc_advance(vd, k4 * 2048),
+                        idesc_pv, (accumulate || half > 0 || k4 > 0) ? 1u : 0u);
+          }
+        };
+        bool ok = true;
+        for (int i = 0; i < n_qt && ok; ++i) ok = ptx::mbar_wait(&q_full[i], 0, abort_flag, a.dev_status);
+        if (ok) ok = ptx::mbar_wait(&kv_full[0], 0, abort_flag, a.dev_status);     // K_0
+        if (ok) {
           ptx::tc_fence_after_sync();
-          issue_pv(i, vslot, j > 0);
-          if (i == n_qt - 1) ptx::mma_commit(&kv_empty[vslot]);
-          if (more) {
-            if (i == 0) ok = ptx::mbar_wait(&kv_full[kslot], (itk / kKvSlots) & 1, abort_flag, a.dev_status);
+          for (int i = 0; i < n_qt; ++i) { issue_qk(i, 0); ptx::mma_commit(&s_full[i]); }
+          ptx::mma_commit(&kv_empty[0]);
+        }
+        for (int j = 0; j < n_kv && ok; ++j) {
+          const int itv = 2 * j + 1, itk = 2 * j + 2;
+          const int vslot = itv % kKvSlots, kslot = itk % kKvSlots;
+          const bool more = j + 1 < n_kv;
+          for (int i = 0; i < n_qt && ok; ++i) {
+            ok = ptx::mbar_wait(&p_lo[i], j & 1, abort_flag, a.dev_status);          // first half of P_j(i), O_i consistent
+            if (ok && i == 0) ok = ptx::mbar_wait(&kv_full[vslot], (itv / kKvSlots) & 1, abort_flag, a.dev_status);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            issue_qk(i, kslot);
-            ptx::mma_commit(&s_full[i]);
-            if (i == n_qt - 1) ptx::mma_commit(&kv_empty[kslot]);
-          } else {
-            ptx::mma_commit(&o_final[i]);
+            issue_pv_half(i, vslot, 0, j > 0);
+            ok = ptx::mbar_wait(&p_hi[i], j & 1, abort_flag, a.dev_status);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            issue_pv_half(i, vslot, 1, true);
+            if (i == n_qt - 1) ptx::mma_commit(&kv_empty[vslot]);
+            if (more) {
+              if (i == 0) ok = ptx::mbar_wait(&kv_full[kslot], (itk / kKvSlots) & 1, abort_flag, a.dev_status);
+              if (!ok) break;
+              ptx::tc_fence_after_sync();
+              issue_qk(i, kslot);
+              ptx::mma_commit(&s_full[i]);
+              if (i == n_qt - 1) ptx::mma_commit(&kv_empty[kslot]);
+            } else {
+              ptx::mma_commit(&o_final[i]);
+            }
           }
         }
       }
     }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
     // ------------------------------------------------------------ softmax + epilogue
     const int i = warp >> 2;                       // query tile of this warpgroup
     const int quarter = warp & 3;
@@ -180,8 +224,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       }
       float* score_row = dec_slot >= 0 ? a.score_scratch + ((size_t)h * a.max_deciders + dec_slot) * a.vis_stride : nullptr;
 
-      float m_used = -INFINITY, l_sum = 0.f;
+      float m_used = -INFINITY;
+      float2 l2 = make_float2(0.f, 0.f);           // the row sum, kept as two partial sums
       const float c = a.scale_log2;
+      const float2 c2 = make_float2(c, c);
       bool ok = true;
       for (int j = 0; j < n_kv; ++j) {
         ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[i], j & 1, abort_flag, a.dev_status));
@@ -199,7 +245,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
           for (int e = 0; e < kTile; ++e) if (e >= n_valid) sr[e] = 0xff800000u;
         }
-        if (score_row != nullptr) {                         // decider row: raw scores over the visual keys
+        if (score_row != nullptr && j * kTile < n_vis) {    // decider row: raw scores over the visual keys
           const int key0 = j * kTile;
 #pragma unroll
           for (int e = 0; e < kTile; e += 4) {
@@ -213,15 +259,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
           }
         }
-        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]), mx2 = __uint_as_float(sr[2]),
-              mx3 = __uint_as_float(sr[3]);
+        // ---- row maximum: 8 independent chains of three-input maxima
+        float mx[8];
 #pragma unroll
-        for (int e = 4; e < kTile; e += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(sr[e]));     mx1 = fmaxf(mx1, __uint_as_float(sr[e + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(sr[e + 2])); mx3 = fmaxf(mx3, __uint_as_float(sr[e + 3]));
-        }
-        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-        const float m_new = fmaxf(m_used, mx * c);
+        for (int t = 0; t < 8; ++t) mx[t] = fmaxf(__uint_as_float(sr[2 * t]), __uint_as_float(sr[2 * t + 1]));
+#pragma unroll
+        for (int e = 16; e < kTile; e += 16)
+#pragma unroll
+          for (int t = 0; t < 8; ++t)
+            mx[t] = max3(mx[t], __uint_as_float(sr[e + 2 * t]), __uint_as_float(sr[e + 2 * t + 1]));
+        const float mxa = max3(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], mx[5]), fmaxf(mx[6], mx[7]));
+        const float m_new = fmaxf(m_used, mxa * c);
         const bool need = (m_new - m_used) > kRescaleThreshold;   // first tile: inf > threshold
         if (__any_sync(0xffffffffu, need)) {
           const float alpha = need ? exp2f(m_used - m_new) : 1.f;
@@ -237,38 +285,45 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
             ptx::tmem_wait_st();
           }
-          l_sum *= alpha;
+          l2.x *= alpha; l2.y *= alpha;
           if (need) m_used = m_new;
         }
-        // ---- p = exp2(s*c - m), row sum, bf16 P tile into the first 64 columns of the S tile
-        const float neg_m = -m_used;
-        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+        // ---- p = exp2(s*c - m) in four chunks of 32 keys; the bf16 P tile goes into the first 64
+        //      columns of the S tile; the tensor pipe is told after each half
+        const float2 nm2 = make_float2(-m_used, -m_used);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t pk[32];
+        for (int ch = 0; ch < 4; ++ch) {
+          float2 t2[16];
 #pragma unroll
-          for (int e = 0; e < 64; e += 4) {
-            const int x = half * 64 + e;
-            const float p0 = ptx::ex2(fmaf(__uint_as_float(sr[x]), c, neg_m));
-            const float p1 = ptx::ex2(fmaf(__uint_as_float(sr[x + 1]), c, neg_m));
-            const float p2 = ptx::ex2(fmaf(__uint_as_float(sr[x + 2]), c, neg_m));
-            const float p3 = ptx::ex2(fmaf(__uint_as_float(sr[x + 3]), c, neg_m));
-            sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
-            __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1), h23 = __floats2bfloat162_rn(p2, p3);
-            pk[e >> 1] = *reinterpret_cast<uint32_t*>(&h01);
-            pk[(e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h23);
+          for (int e = 0; e < 16; ++e)
+            t2[e] = __ffma2_rn(make_float2(__uint_as_float(sr[ch * 32 + 2 * e]), __uint_as_float(sr[ch * 32 + 2 * e + 1])),
+                               c2, nm2);
+#pragma unroll
+          for (int e = 0; e < 16; ++e) { t2[e].x = ptx::ex2(t2[e].x); t2[e].y = ptx::ex2(t2[e].y); }
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            pk[e] = pack_bf16x2(t2[e].x, t2[e].y);
+            l2 = __fadd2_rn(l2, t2[e]);
           }
-          ptx::tmem_st32(t_s + half * 32, pk);             // keys 64*half .. +63 -> P columns 32*half .. +31
+          if (ch == 2) {                                   // the first half has been stored two chunks ago
+            ptx::tmem_wait_st();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&p_lo[i]);
+          }
+          tmem_st16(t_s + ch * 16, pk);                    // keys 32*ch .. +31 -> P columns 16*ch .. +15
         }
-        l_sum += (sum0 + sum1) + (sum2 + sum3);
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
-        ptx::mbar_arrive(&p_full[i]);
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&p_hi[i]);
       }
       // ---- epilogue: O / l -> bf16 -> global
       if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&o_final[i], 0, abort_flag, a.dev_status));
       ptx::tc_fence_after_sync();
       if (ok) {
+        const float l_sum = l2.x + l2.y;
         const float inv_l = 1.f / l_sum;
         __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(a.out) + ((size_t)(lo + q_row) * a.H + h) * DH;
 #pragma unroll 1
@@ -281,11 +336,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             for (int e = 0; e < 32; e += 8) {
               uint32_t w[4];
 #pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[e + 2 * t]) * inv_l,
-                                                          __uint_as_float(r[e + 2 * t + 1]) * inv_l);
-                w[t] = *reinterpret_cast<uint32_t*>(&h2);
-              }
+              for (int t = 0; t < 4; ++t)
+                w[t] = pack_bf16x2(__uint_as_float(r[e + 2 * t]) * inv_l, __uint_as_float(r[e + 2 * t + 1]) * inv_l);
               *reinterpret_cast<uint4*>(dst + c0 + e) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }

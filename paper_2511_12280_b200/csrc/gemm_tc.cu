@@ -102,17 +102,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, BN, 0, 0);
+      const ptx::SmemDesc a_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(a_s));
+      const ptx::SmemDesc b_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(b_s));
       bool ok = true;
       for (int kbk = 0; kbk < p.num_k_blocks && ok; ++kbk) {
         const int s = kbk % kStages;
         ok = ptx::mbar_wait(&full[s], (kbk / kStages) & 1, abort_flag, p.dev_status);
         if (!ok) break;
         ptx::tc_fence_after_sync();
-        const uint32_t a_addr = ptx::smem_u32(a_s + s * S::kABytes), b_addr = ptx::smem_u32(b_s + s * S::kBBytes);
+        const ptx::SmemDesc ad = ptx::smem_desc_advance(a_desc0, s * S::kABytes), bd = ptx::smem_desc_advance(b_desc0, s * S::kBBytes);
 #pragma unroll
         for (int kk = 0; kk < kBK / 16; ++kk) {
-          ptx::mma_ss(tmem_acc, ptx::smem_desc_kmajor_sw128(a_addr + kk * 32), ptx::smem_desc_kmajor_sw128(b_addr + kk * 32),
-                      idesc, (kbk > 0 || kk > 0) ? 1u : 0u);
+          ptx::mma_ss(tmem_acc, ptx::smem_desc_advance(ad, kk * 32), ptx::smem_desc_advance(bd, kk * 32), idesc,
+                      (kbk > 0 || kk > 0) ? 1u : 0u);
         }
         ptx::mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
       }

@@ -106,22 +106,31 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {  
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// A shared-memory matrix descriptor is handled as two 32-bit halves so that moving
+// along a tile costs one 32-bit add per tcgen05.mma: the issuing thread's own
+// instruction stream, not the tensor pipe, limits 128 x 128 x 16 instructions
+// (64 cycles each) as soon as it spends more than a few instructions per MMA.
+struct SmemDesc { uint32_t lo, hi; };
+
 // D[tmem] (+)= A[smem] * B[smem]; one thread issues.
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, SmemDesc a, SmemDesc b, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a.lo), "r"(a.hi), "r"(b.lo), "r"(b.hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, SmemDesc b, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b.lo), "r"(b.hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // arrive on `bar` once every tcgen05.mma issued so far by this thread has completed
@@ -174,16 +183,27 @@ __device__ __forceinline__ float ex2(float x) {
 //   bits 61..63  swizzle mode (2 = 128 B)
 // K-major operand (rows x 64 bf16, 128-byte rows): 8-row groups are 1024 B apart
 // (SBO); LBO is unused.  Advancing K by 16 elements adds 32 bytes to the start.
-__device__ __forceinline__ uint64_t smem_desc_kmajor_sw128(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
-         (2ull << 61);
+// The two 32-bit halves: lo = start | LBO << 16, hi = SBO | version << 14 | swizzle << 29.
+__device__ __forceinline__ SmemDesc smem_desc_kmajor_sw128(uint32_t smem_addr) {
+  SmemDesc d;
+  d.lo = ((smem_addr >> 4) & 0x3fffu) | (1u << 16);
+  d.hi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+  return d;
 }
 // MN-major operand (K rows of 128 bytes = 64 bf16 along MN): 8-row groups along K
 // are 1024 B apart (SBO); consecutive 64-element blocks along MN are lbo_bytes
 // apart (LBO).  Advancing K by 16 rows adds 2048 bytes to the start.
-__device__ __forceinline__ uint64_t smem_desc_mnmajor_sw128(uint32_t smem_addr, uint32_t lbo_bytes) {
-  return (uint64_t)((smem_addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
-         ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+__device__ __forceinline__ SmemDesc smem_desc_mnmajor_sw128(uint32_t smem_addr, uint32_t lbo_bytes) {
+  SmemDesc d;
+  d.lo = ((smem_addr >> 4) & 0x3fffu) | (((lbo_bytes >> 4) & 0x3fffu) << 16);
+  d.hi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+  return d;
+}
+// The same descriptor with its start moved by `bytes` (a multiple of 16; the start field is
+// 14 bits of 16-byte units and shared-memory addresses stay below 256 KB, so no carry leaves it).
+__device__ __forceinline__ SmemDesc smem_desc_advance(SmemDesc d, uint32_t bytes) {
+  d.lo += bytes >> 4;
+  return d;
 }
 // Instruction descriptor, kind::f16, bf16 x bf16 -> fp32:
 //   bits 4..5 D type (1 = f32), 7..9 A type (1 = bf16), 10..12 B type (1 = bf16),
