@@ -10,7 +10,7 @@
 // ping-pong on the tensor pipe.
 //   warps 0-3   softmax of query tile 0 (one row per thread = one TMEM lane)
 //   warps 4-7   softmax of query tile 1
-//   warp  8     TMA producer: Q tiles once, then K_j / V_j tiles through a ring
+//   warp  8     TMA producer: Q tiles once, then stages {K_t, V_(t-1)}, two in flight
 //   warp  9     one thread issues every tcgen05.mma
 //   warps 10-11 idle (they complete the third warpgroup so that registers can be
 //               moved from it to the softmax warpgroups with setmaxnreg)
@@ -78,11 +78,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;                                  // 2 tiles
-  uint8_t* kv_s = smem + 2 * kTileBytes;                // ring: K_0, V_0, K_1, V_1, ...
+  uint8_t* kv_s = smem + 2 * kTileBytes;                // two stages of {K tile, V tile}
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (2 + kKvSlots) * kTileBytes);
   uint64_t* q_full = bars;                              // [2]
-  uint64_t* kv_full = bars + 2;                         // [4]
-  uint64_t* kv_empty = bars + 6;                        // [4]
+  uint64_t* kv_full = bars + 2;                         // [2] (of 4 reserved)
+  uint64_t* kv_empty = bars + 6;                        // [2] (of 4 reserved)
   uint64_t* s_full = bars + 10;                         // [2]
   uint64_t* p_lo = bars + 12;                           // [2]  P columns of keys 0..63 written (and O consistent)
   uint64_t* p_hi = bars + 14;                           // [2]  P columns of keys 64..127 written
@@ -122,14 +122,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             ptx::tma_load_2d(q_s + i * kTileBytes + hf * kHalfBytes, &tmap_q, &q_full[i], h * DH + hf * 64,
                              lo + q0 + i * kTile);
         }
-        for (int it = 0; it < 2 * n_kv; ++it) {             // it = 2j: K_j, it = 2j+1: V_j
-          const int slot = it % kKvSlots, j = it >> 1;
-          if (!ptx::mbar_wait(&kv_empty[slot], ((it / kKvSlots) & 1) ^ 1, abort_flag, a.dev_status)) break;
-          ptx::mbar_arrive_expect_tx(&kv_full[slot], kTileBytes);
-          const CUtensorMap* tm = (it & 1) ? &tmap_v : &tmap_k;
-          for (int hf = 0; hf < kHalves; ++hf)
-            ptx::tma_load_2d(kv_s + slot * kTileBytes + hf * kHalfBytes, tm, &kv_full[slot], h * DH + hf * 64,
-                             lo + j * kTile);
+        // stage t = {K_t, V_(t-1)}: what key tile t-1's PV and key tile t's QK^T need; two stages in flight
+        for (int t = 0; t <= n_kv; ++t) {
+          const int st = t & 1;
+          if (t >= 2 && !ptx::mbar_wait(&kv_empty[st], ((t >> 1) & 1) ^ 1, abort_flag, a.dev_status)) break;
+          const bool has_k = t < n_kv, has_v = t > 0;
+          ptx::mbar_arrive_expect_tx(&kv_full[st], (has_k ? kTileBytes : 0) + (has_v ? kTileBytes : 0));
+          for (int hf = 0; hf < kHalves; ++hf) {
+            if (has_v) ptx::tma_load_2d(kv_s + (2 * st + 1) * kTileBytes + hf * kHalfBytes, &tmap_v, &kv_full[st],
+                                        h * DH + hf * 64, lo + (t - 1) * kTile);
+            if (has_k) ptx::tma_load_2d(kv_s + (2 * st) * kTileBytes + hf * kHalfBytes, &tmap_k, &kv_full[st],
+                                        h * DH + hf * 64, lo + t * kTile);
+          }
         }
       }
     } else if (warp == 9) {
@@ -164,38 +168,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         };
         bool ok = true;
         for (int i = 0; i < n_qt && ok; ++i) ok = ptx::mbar_wait(&q_full[i], 0, abort_flag, a.dev_status);
-        if (ok) ok = ptx::mbar_wait(&kv_full[0], 0, abort_flag, a.dev_status);     // K_0
+        if (ok) ok = ptx::mbar_wait(&kv_full[0], 0, abort_flag, a.dev_status);     // stage 0 = K_0
         if (ok) {
           ptx::tc_fence_after_sync();
           for (int i = 0; i < n_qt; ++i) { issue_qk(i, 0); ptx::mma_commit(&s_full[i]); }
-          ptx::mma_commit(&kv_empty[0]);
+          ptx::mma_commit(&kv_empty[0]);          // stage 0 held K_0 only: the producer may go on to stage 2
         }
+        // Key tile j needs stage j+1 (V_j and K_(j+1)).  The softmax warps wait for that stage
+        // before they announce P_j, so this thread has no load barrier of its own to check: every
+        // barrier check between two MMAs costs the tensor pipe more than an instruction slot.
         for (int j = 0; j < n_kv && ok; ++j) {
-          const int itv = 2 * j + 1, itk = 2 * j + 2;
-          const int vslot = itv % kKvSlots, kslot = itk % kKvSlots;
+          const int st = (j + 1) & 1;
           const bool more = j + 1 < n_kv;
           for (int i = 0; i < n_qt && ok; ++i) {
             ok = ptx::mbar_wait(&p_lo[i], j & 1, abort_flag, a.dev_status);          // first half of P_j(i), O_i consistent
-            if (ok && i == 0) ok = ptx::mbar_wait(&kv_full[vslot], (itv / kKvSlots) & 1, abort_flag, a.dev_status);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            issue_pv_half(i, vslot, 0, j > 0);
+            issue_pv_half(i, 2 * st + 1, 0, j > 0);
             ok = ptx::mbar_wait(&p_hi[i], j & 1, abort_flag, a.dev_status);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            issue_pv_half(i, vslot, 1, true);
-            if (i == n_qt - 1) ptx::mma_commit(&kv_empty[vslot]);
+            issue_pv_half(i, 2 * st + 1, 1, true);
             if (more) {
-              if (i == 0) ok = ptx::mbar_wait(&kv_full[kslot], (itk / kKvSlots) & 1, abort_flag, a.dev_status);
-              if (!ok) break;
-              ptx::tc_fence_after_sync();
-              issue_qk(i, kslot);
+              issue_qk(i, 2 * st);
               ptx::mma_commit(&s_full[i]);
-              if (i == n_qt - 1) ptx::mma_commit(&kv_empty[kslot]);
             } else {
               ptx::mma_commit(&o_final[i]);
             }
           }
+          if (ok) ptx::mma_commit(&kv_empty[st]);   // frees stage j+1 once everything issued so far is done
         }
       }
     }
@@ -309,11 +310,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           if (ch == 2) {                                   // the first half has been stored two chunks ago
             ptx::tmem_wait_st();
             ptx::tc_fence_before_sync();
-            __syncwarp();
+            // V_j and K_(j+1) must have landed before the tensor pipe is sent on (it does not check)
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&kv_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag, a.dev_status));
+            if (!ok) break;
             if (lane == 0) ptx::mbar_arrive(&p_lo[i]);
           }
           tmem_st16(t_s + ch * 16, pk);                    // keys 32*ch .. +31 -> P columns 16*ch .. +15
         }
+        if (!ok) break;
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
         __syncwarp();
