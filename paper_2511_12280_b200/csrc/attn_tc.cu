@@ -246,20 +246,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
           for (int e = 0; e < kTile; ++e) if (e >= n_valid) sr[e] = 0xff800000u;
         }
-        if (score_row != nullptr && j * kTile < n_vis) {    // decider row: raw scores over the visual keys
-          const int key0 = j * kTile;
+        // ---- p = exp2(s*c - m) in four chunks of 32 keys.  The first two chunks are computed
+        //      against the maximum known BEFORE this tile, while the tile's own maximum is still being
+        //      reduced: any reference within 2^8 of the true maximum is exact after the final division,
+        //      so the result stands unless the maximum grew by more than that (then it is redone).
+        uint32_t pk[2][16];
+        float2 l_tile = make_float2(0.f, 0.f);
+        auto exp_chunk = [&](int ch, float m_ref, uint32_t (&out)[16], float2& lsum) {
+          const float2 nm2 = make_float2(-m_ref, -m_ref);
+          float2 t2[16];
 #pragma unroll
-          for (int e = 0; e < kTile; e += 4) {
-            if (key0 + e + 3 < n_vis) {
-              *reinterpret_cast<float4*>(score_row + key0 + e) =
-                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
-                              __uint_as_float(sr[e + 3]));
-            } else {
+          for (int e = 0; e < 16; ++e)
+            t2[e] = __ffma2_rn(make_float2(__uint_as_float(sr[ch * 32 + 2 * e]), __uint_as_float(sr[ch * 32 + 2 * e + 1])),
+                               c2, nm2);
 #pragma unroll
-              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
-            }
+          for (int e = 0; e < 16; ++e) { t2[e].x = ptx::ex2(t2[e].x); t2[e].y = ptx::ex2(t2[e].y); }
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            out[e] = pack_bf16x2(t2[e].x, t2[e].y);
+            lsum = __fadd2_rn(lsum, t2[e]);
           }
-        }
+        };
+        exp_chunk(0, m_used, pk[0], l_tile);                // (first tile: against -inf, always redone below)
+        exp_chunk(1, m_used, pk[1], l_tile);
         // ---- row maximum: 8 independent chains of three-input maxima
         float mx[8];
 #pragma unroll
@@ -288,36 +297,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           }
           l2.x *= alpha; l2.y *= alpha;
           if (need) m_used = m_new;
+          l_tile = make_float2(0.f, 0.f);                   // the speculative half is redone against the new maximum
+          exp_chunk(0, m_used, pk[0], l_tile);
+          exp_chunk(1, m_used, pk[1], l_tile);
         }
-        // ---- p = exp2(s*c - m) in four chunks of 32 keys; the bf16 P tile goes into the first 64
-        //      columns of the S tile; the tensor pipe is told after each half
-        const float2 nm2 = make_float2(-m_used, -m_used);
+        if (score_row != nullptr && j * kTile < n_vis) {    // decider row: raw scores over the visual keys
+          const int key0 = j * kTile;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          float2 t2[16];
+          for (int e = 0; e < kTile; e += 4) {
+            if (key0 + e + 3 < n_vis) {
+              *reinterpret_cast<float4*>(score_row + key0 + e) =
+                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
+                              __uint_as_float(sr[e + 3]));
+            } else {
 #pragma unroll
-          for (int e = 0; e < 16; ++e)
-            t2[e] = __ffma2_rn(make_float2(__uint_as_float(sr[ch * 32 + 2 * e]), __uint_as_float(sr[ch * 32 + 2 * e + 1])),
-                               c2, nm2);
-#pragma unroll
-          for (int e = 0; e < 16; ++e) { t2[e].x = ptx::ex2(t2[e].x); t2[e].y = ptx::ex2(t2[e].y); }
-          uint32_t pk[16];
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            pk[e] = pack_bf16x2(t2[e].x, t2[e].y);
-            l2 = __fadd2_rn(l2, t2[e]);
+              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
+            }
           }
-          if (ch == 2) {                                   // the first half has been stored two chunks ago
-            ptx::tmem_wait_st();
-            ptx::tc_fence_before_sync();
-            // V_j and K_(j+1) must have landed before the tensor pipe is sent on (it does not check)
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&kv_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag, a.dev_status));
-            if (!ok) break;
-            if (lane == 0) ptx::mbar_arrive(&p_lo[i]);
-          }
-          tmem_st16(t_s + ch * 16, pk);                    // keys 32*ch .. +31 -> P columns 16*ch .. +15
         }
+        // ---- the bf16 P tile goes into the first 64 columns of the S tile; the tensor pipe is told after each half
+        tmem_st16(t_s, pk[0]);                             // keys 32*ch .. +31 -> P columns 16*ch .. +15
+        tmem_st16(t_s + 16, pk[1]);
+        exp_chunk(2, m_used, pk[0], l_tile);
+        ptx::tmem_wait_st();
+        ptx::tc_fence_before_sync();
+        // V_j and K_(j+1) must have landed before the tensor pipe is sent on (it does not check)
+        ok = __all_sync(0xffffffffu, ptx::mbar_wait(&kv_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag, a.dev_status));
         if (!ok) break;
+        if (lane == 0) ptx::mbar_arrive(&p_lo[i]);
+        tmem_st16(t_s + 32, pk[0]);
+        exp_chunk(3, m_used, pk[1], l_tile);
+        tmem_st16(t_s + 48, pk[1]);
+        l2 = __fadd2_rn(l2, l_tile);
         ptx::tmem_wait_st();
         ptx::tc_fence_before_sync();
         __syncwarp();
