@@ -137,8 +137,9 @@ int d3tom_attn_importance(d3tom_ctx* ctx, d3tom_dtype dt,
  *     heads * max(1, n_deciders_total)                       <= D3TOM_STATIC_MAX_LSE_PAIRS
  *     heads * total_tokens                                   <= D3TOM_STATIC_MAX_PARTIAL_FLOATS
  *     heads * max(1, n_deciders_total) * round_up(max_visual, 4) <= D3TOM_STATIC_MAX_SCORE_FLOATS
- * returns D3TOM_ERR_WORKSPACE and launches nothing (e.g. 32 heads x 16
- * deciders x 4096 visual tokens, 16384 packed tokens, fits exactly).
+ * (or with B * ceil(max_visual / 256) > 4096) returns D3TOM_ERR_WORKSPACE and
+ * launches nothing (e.g. 32 heads x 16 deciders x 4096 visual tokens, 16384
+ * packed tokens, fits exactly).
  *
  * heads, head_dim replace the context's limits; every other argument is as in
  * d3tom_attn_importance, and the results are the same bit for bit.  The work
@@ -150,7 +151,7 @@ int d3tom_attn_importance(d3tom_ctx* ctx, d3tom_dtype dt,
  * The first call on each device looks up the array's device address; make
  * that first call outside of any stream capture.  No call allocates or frees.
  * All calls on a device share the one array, and it keeps what the previous
- * call left there (this function clears the only word that has to start at
+ * call left there (this function clears the few words that have to start at
  * zero): two calls that overlap on the GPU race with each other, so keep all
  * calls of a device on one stream or order them with events. */
 #define D3TOM_STATIC_MAX_LSE_PAIRS      (1 << 14)

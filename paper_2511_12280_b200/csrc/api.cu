@@ -26,7 +26,8 @@ int alloc(d3tom_ctx* ctx, T** p, size_t count) {
 }
 
 void free_all(d3tom_ctx* c) {
-  cudaFree(c->score_scratch); cudaFree(c->lse_scratch); cudaFree(c->imp_partial); cudaFree(c->inv_norm);
+  cudaFree(c->score_scratch); cudaFree(c->lse_scratch); cudaFree(c->imp_partial); cudaFree(c->imp_counters);
+  cudaFree(c->inv_norm);
   cudaFree(c->inv_norm_kept); cudaFree(c->kept_rows); cudaFree(c->best); cudaFree(c->member_off);
   cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->dev_status);
 }
@@ -69,6 +70,9 @@ int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (st == D3TOM_OK) st = alloc(c, &c->score_scratch, H * nd * c->vis_stride);
   if (st == D3TOM_OK) st = alloc(c, &c->lse_scratch, H * nd);
   if (st == D3TOM_OK) st = alloc(c, &c->imp_partial, H * T);
+  const size_t n_ctr = (size_t)lim->max_batch * (((size_t)lim->max_visual_per_request + 255) / 256);
+  if (st == D3TOM_OK) st = alloc(c, &c->imp_counters, n_ctr);
+  if (st == D3TOM_OK && cudaMemset(c->imp_counters, 0, n_ctr * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st == D3TOM_OK) st = alloc(c, &c->inv_norm, T);
   if (st == D3TOM_OK) st = alloc(c, &c->inv_norm_kept, T);
   if (st == D3TOM_OK) st = alloc(c, reinterpret_cast<char**>(&c->kept_rows), T * D * sizeof(float));

@@ -8,7 +8,7 @@
 //
 // Decider rows additionally write their raw q.k scores over the visual keys to
 // the score scratch and their final (M, l) pair to the lse scratch; the
-// finishing kernels turn those into S_j = sum_h sum_{i in D} A_ij.
+// finishing kernel turns those into S_j = sum_h sum_{i in D} A_ij.
 #include "common.cuh"
 
 namespace {
@@ -87,35 +87,61 @@ attn_simt_kernel(AttnArgs a) {
   if (dec_slot >= 0 && lane == 0) a.lse_scratch[(size_t)h * a.max_deciders + dec_slot] = make_float2(m, l);
 }
 
-// partial[h][cu_vis[b] + j] = sum over the request's deciders (ascending) of
-// exp2(score * c - M) / l
-__global__ void __launch_bounds__(256)
-importance_partial_kernel(const float* __restrict__ score, const float2* __restrict__ lse,
-                          const int32_t* __restrict__ n_visual, const int32_t* __restrict__ cu_deciders,
-                          const int32_t* __restrict__ cu_vis, int max_deciders, int vis_stride,
-                          float scale_log2, float* __restrict__ partial, int partial_stride) {
-  const int b = blockIdx.z, h = blockIdx.y;
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= n_visual[b]) return;
-  const int d0 = cu_deciders[b], d1 = cu_deciders[b + 1];
-  float acc = 0.f;
-  for (int d = d0; d < d1; ++d) {
-    const size_t r = (size_t)h * max_deciders + d;
-    const float2 ml = lse[r];
-    acc += exp2f(fmaf(score[r * vis_stride + j], scale_log2, -ml.x)) / ml.y;
-  }
-  partial[(size_t)h * partial_stride + cu_vis[b] + j] = acc;
-}
+// One block = (256 visual keys, head, request).
+//   partial[h][cu_vis[b] + j] = sum over the request's deciders (ascending) of exp2(score * c - M) / l
+// The last of the H blocks of a key range to finish (a counter per range, left at zero again
+// afterwards) adds the H partials in ascending head order:
+//   importance[g] = sum over heads of partial[h][g]
+// so the result does not depend on which block that is: no float atomics, reproducible.
+constexpr int kImpThreads = 256;
+constexpr int kImpDecChunk = 128;
 
-// importance[g] = sum over heads (ascending) of partial[h][g]
-__global__ void __launch_bounds__(256)
-importance_reduce_kernel(const float* __restrict__ partial, int partial_stride, int H,
-                         const int32_t* __restrict__ cu_vis, int B, float* __restrict__ importance) {
-  const int g = blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= cu_vis[B]) return;
+__global__ void __launch_bounds__(kImpThreads)
+importance_finish_kernel(const float* __restrict__ score, const float2* __restrict__ lse,
+                         const int32_t* __restrict__ n_visual, const int32_t* __restrict__ cu_deciders,
+                         const int32_t* __restrict__ cu_vis, int max_deciders, int vis_stride, float scale_log2,
+                         float* __restrict__ partial, int partial_stride, int H, int* __restrict__ counters,
+                         float* __restrict__ importance) {
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int Vb = n_visual[b];
+  if ((int)blockIdx.x * kImpThreads >= Vb) return;              // uniform: no key of this request in the range
+  const int j = blockIdx.x * kImpThreads + threadIdx.x;
+  const int d0 = cu_deciders[b], d1 = cu_deciders[b + 1];
+  __shared__ float neg_m[kImpDecChunk], inv_l[kImpDecChunk];
+  __shared__ int is_last;
+  const int jj = j < Vb ? j : Vb - 1;                           // threads past the end read a valid column, write nothing
   float acc = 0.f;
-  for (int h = 0; h < H; ++h) acc += partial[(size_t)h * partial_stride + g];
-  importance[g] = acc;
+  for (int dc = d0; dc < d1; dc += kImpDecChunk) {
+    const int nd = min(kImpDecChunk, d1 - dc);
+    __syncthreads();
+    if (threadIdx.x < nd) {
+      const float2 ml = lse[(size_t)h * max_deciders + dc + threadIdx.x];
+      neg_m[threadIdx.x] = -ml.x;
+      inv_l[threadIdx.x] = 1.0f / ml.y;
+    }
+    __syncthreads();
+    const float* col = score + ((size_t)h * max_deciders + dc) * vis_stride + jj;
+#pragma unroll 8
+    for (int d = 0; d < nd; ++d)
+      acc = fmaf(exp2f(fmaf(col[(size_t)d * vis_stride], scale_log2, neg_m[d])), inv_l[d], acc);
+  }
+  const int g0 = cu_vis[b];
+  if (j < Vb) partial[(size_t)h * partial_stride + g0 + j] = acc;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int* ctr = counters + (size_t)b * gridDim.x + blockIdx.x;
+    const int prev = atomicAdd(ctr, 1);
+    is_last = prev == H - 1;
+    if (is_last) *ctr = 0;                                      // ready for the next call
+  }
+  __syncthreads();
+  if (is_last && j < Vb) {
+    __threadfence();
+    float tot = 0.f;
+    for (int hh = 0; hh < H; ++hh) tot += __ldcg(partial + (size_t)hh * partial_stride + g0 + j);
+    importance[g0 + j] = tot;
+  }
 }
 
 }  // namespace
@@ -131,15 +157,10 @@ int launch_attn_simt(d3tom_ctx* ctx, d3tom_dtype dt, const AttnArgs& a, cudaStre
 int launch_importance_finish(d3tom_ctx* ctx, const AttnArgs& a, int max_visual, float* importance,
                              const int32_t* cu_vis, cudaStream_t s) {
   if (max_visual <= 0) return D3TOM_OK;
-  dim3 grid(ceil_div(max_visual, 256), a.H, a.B);
-  importance_partial_kernel<<<grid, 256, 0, s>>>(a.score_scratch, a.lse_scratch, a.n_visual, a.cu_deciders, cu_vis,
-                                                 a.max_deciders, a.vis_stride, a.scale_log2, ctx->imp_partial,
-                                                 ctx->lim.max_total_tokens);
-  D3TOM_LAUNCH_CHECK(ctx);
-  // the visual total is cu_vis[B] on the device; the grid is sized by its host bound
-  const int total_vis_bound = min(a.total_tokens, a.B * max_visual);
-  importance_reduce_kernel<<<ceil_div(total_vis_bound, 256), 256, 0, s>>>(ctx->imp_partial, ctx->lim.max_total_tokens,
-                                                                          a.H, cu_vis, a.B, importance);
+  dim3 grid(ceil_div(max_visual, kImpThreads), a.H, a.B);
+  importance_finish_kernel<<<grid, kImpThreads, 0, s>>>(a.score_scratch, a.lse_scratch, a.n_visual, a.cu_deciders, cu_vis,
+                                                        a.max_deciders, a.vis_stride, a.scale_log2, ctx->imp_partial,
+                                                        ctx->lim.max_total_tokens, a.H, ctx->imp_counters, importance);
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }

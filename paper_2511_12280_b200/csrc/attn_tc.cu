@@ -68,9 +68,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   constexpr int kTileBytes = S::kTileBytes;
   constexpr int kHalfBytes = kTile * 128;               // one 64-column sub-tile: 128 rows x 128 bytes
   constexpr int kHalves = DH / 64;
-  const int b = blockIdx.z, h = blockIdx.y;
+  // CTAs of a request are dispatched in the order of their linear index (x fastest).  The first H
+  // indices take the LAST 256-row query block of every head: the response rows live there and
+  // decider rows do extra work, so those CTAs must not end up in the last wave.  The remaining
+  // indices walk head by head (one head's K/V stay hot in L2), query blocks from the end.
+  const int b = blockIdx.z;
+  const int linear = (int)blockIdx.y * (int)gridDim.x + (int)blockIdx.x, nqb = (int)gridDim.x;
+  int h, qb;
+  if (linear < a.H) { h = linear; qb = nqb - 1; }
+  else { const int r = linear - a.H; h = r / (nqb - 1); qb = nqb - 2 - r % (nqb - 1); }
   const int lo = a.cu_seqlens[b], n = a.cu_seqlens[b + 1] - lo;
-  const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * 2 * kTile;   // last rows of the request first
+  const int q0 = qb * 2 * kTile;
   if (q0 >= n) return;                                  // uniform; nothing allocated yet
   const int n_qt = (n - q0 > kTile) ? 2 : 1;
   const int n_kv = (n + kTile - 1) / kTile;

@@ -18,6 +18,7 @@ struct d3tom_ctx {
   float* score_scratch;         // [H][max_deciders][vis_stride] raw q.k of decider rows x visual keys
   float2* lse_scratch;          // [H][max_deciders] (M, l): l = sum_j exp2(s_j*c - M)
   float* imp_partial;           // [H][max_total_tokens] per-head importance
+  int* imp_counters;            // [max_batch][ceil(max_visual / 256)] blocks done per key range; zero between calls
   float* inv_norm;              // [max_total_tokens] 1/|h| of visual rows (packed by cu_vis)
   float* inv_norm_kept;         // [max_total_tokens] the same for kept rows, packed by cu_kept
   void* kept_rows;              // [max_total_tokens, D] gathered kept rows (B operand of the similarity GEMM)

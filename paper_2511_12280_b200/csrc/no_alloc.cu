@@ -18,8 +18,9 @@
 
 namespace {
 
-// layout of the array (bytes): [status word | (M, l) pairs | per-head partials | raw decider scores]
-constexpr size_t kStatusBytes = 256;
+// layout of the array (bytes): [status word + key-range counters | (M, l) pairs | per-head partials | raw decider scores]
+constexpr size_t kCounterInts = 4096;     // batch * ceil(max_visual / 256) must stay below this
+constexpr size_t kStatusBytes = 256 + kCounterInts * sizeof(int);
 constexpr size_t kLseBytes = (size_t)D3TOM_STATIC_MAX_LSE_PAIRS * sizeof(float2);
 constexpr size_t kPartialBytes = (size_t)D3TOM_STATIC_MAX_PARTIAL_FLOATS * sizeof(float);
 constexpr size_t kScoreBytes = (size_t)D3TOM_STATIC_MAX_SCORE_FLOATS * sizeof(float);
@@ -81,7 +82,8 @@ extern "C" int d3tom_attn_importance_static(d3tom_dtype dt, int heads, int head_
   const size_t vis_stride = ((size_t)max_visual + 3) & ~(size_t)3;
   if ((size_t)heads * nd > (size_t)D3TOM_STATIC_MAX_LSE_PAIRS ||
       (size_t)heads * (size_t)total_tokens > (size_t)D3TOM_STATIC_MAX_PARTIAL_FLOATS ||
-      (size_t)heads * nd * vis_stride > (size_t)D3TOM_STATIC_MAX_SCORE_FLOATS)
+      (size_t)heads * nd * vis_stride > (size_t)D3TOM_STATIC_MAX_SCORE_FLOATS ||
+      (size_t)B * (((size_t)max_visual + 255) / 256) > kCounterInts)
     return D3TOM_ERR_WORKSPACE;
   if (total_tokens == 0 || max_seqlen == 0) return D3TOM_OK;
 
@@ -98,13 +100,14 @@ extern "C" int d3tom_attn_importance_static(d3tom_dtype dt, int heads, int head_
   c.lim.max_deciders = (int)nd; c.lim.max_visual_per_request = max_visual;
   c.vis_stride = (int)vis_stride;
   c.dev_status = reinterpret_cast<int*>(base);
+  c.imp_counters = reinterpret_cast<int*>(base + 256);
   c.lse_scratch = reinterpret_cast<float2*>(base + kStatusBytes);
   c.imp_partial = reinterpret_cast<float*>(base + kStatusBytes + kLseBytes);
   c.score_scratch = reinterpret_cast<float*>(base + kStatusBytes + kLseBytes + kPartialBytes);
 
-  // the array keeps whatever the previous call left: the status word is the one thing that must start at zero
-  // (scores, (M, l) pairs and partials are fully rewritten before they are read)
-  if (cudaMemsetAsync(c.dev_status, 0, sizeof(int), s) != cudaSuccess) return D3TOM_ERR_CUDA;
+  // the array keeps whatever the previous call left: the status word and the key-range counters must start at
+  // zero (scores, (M, l) pairs and partials are fully rewritten before they are read)
+  if (cudaMemsetAsync(base, 0, kStatusBytes, s) != cudaSuccess) return D3TOM_ERR_CUDA;
 
   AttnArgs a;
   a.q = q; a.k = k; a.v = v; a.out = attn_out;

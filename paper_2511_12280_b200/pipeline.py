@@ -116,8 +116,8 @@ class MergeLayerStep:
         return x
 
     def launches_per_step(self) -> int:
-        """Kernels of this library launched by one run(): attention 1 + importance finish 2,
+        """Kernels of this library launched by one run(): attention 1 + importance finish 1,
         select 1, merge 3 (prepare) + 1 (similarity, when something is pruned) + 2 (finish),
         and 2 per post-merge layer."""
         sim = 1 if self.total_out < self.total else 0
-        return 3 + 1 + 3 + sim + 2 + 2 * self.n_post
+        return 2 + 1 + 3 + sim + 2 + 2 * self.n_post
