@@ -155,7 +155,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int g = v0 + m;
         const bool active = m < Vb && p.assign[g] < 0;     // a pruned token of this request
         const float inm = active ? p.inv_norm[g] : 0.f;
-        unsigned long long mine = 0ull;
+        float best_sim = -INFINITY;                        // strict > below: the lowest slot wins a tie
+        int best_slot = 0;
         float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + n0 : nullptr;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
@@ -167,15 +168,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (int i = 0; i < 32; ++i) {
               const int sidx = n0 + c + i;
               if (sidx < kb) {
-                const float sim = (__uint_as_float(r[i]) * inm) * ink_s[c + i];   // the value the arg-max compares
-                const unsigned long long packed =
-                    ((unsigned long long)ordered_key(sim) << 32) | (0xffffffffu - (unsigned)sidx);
-                mine = packed > mine ? packed : mine;
+                // the value the arg-max compares; + 0 turns a negative zero into the positive one
+                const float sim = (__uint_as_float(r[i]) * inm) * ink_s[c + i] + 0.0f;
+                if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
                 if (dbg != nullptr) dbg[c + i] = sim;
               }
             }
           }
         }
+        const unsigned long long mine =
+            ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
         if (active) atomicMax(p.best + g, mine);
       }
     }
@@ -263,5 +265,10 @@ int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   p.cu_seqlens = a.cu_seqlens; p.cu_vis = a.cu_vis; p.cu_kept = a.cu_kept; p.assign = a.assign;
   p.inv_norm = ctx->inv_norm; p.inv_norm_kept = ctx->inv_norm_kept; p.best = ctx->best; p.sim_debug = a.sim_debug;
   p.max_kept = a.max_kept; p.dev_status = ctx->dev_status;
+  if (a.max_kept > 128) {      // 256-wide tiles: the A tile is streamed once per 256 kept rows and each MMA covers twice the work
+    r = make_tmap_bf16_2d(&tb, ctx->kept_rows, (uint64_t)kept_rows_bound, (uint64_t)a.D, (uint64_t)a.D, 256);
+    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+    return launch_gemm<256, kEpiSim>(ctx, ta, tb, p, dim3(ceil_div(a.max_visual, kBM), ceil_div(a.max_kept, 256), a.B), s);
+  }
   return launch_gemm<128, kEpiSim>(ctx, ta, tb, p, dim3(ceil_div(a.max_visual, kBM), ceil_div(a.max_kept, 128), a.B), s);
 }

@@ -2,8 +2,9 @@
 // the removal of the merged positions), everything except the tensor-core
 // similarity kernel:
 //
-//   prepare   slot of every kept token, 1/|h| of every visual row, and a packed
-//             copy of the kept rows (the second operand of the similarity)
+//   prepare   slot of every visual token in the kept list (-1 = pruned), 1/|h| of
+//             every visual row, and a packed copy of the kept rows (the second
+//             operand of the similarity)
 //   sim_simt  cosine + arg-max on CUDA cores (fp32 storage, debugging aid)
 //   finish    destination slots, per-slot member lists, aggregation in
 //             ascending member order and compaction into the shortened sequence
@@ -16,48 +17,52 @@
 namespace {
 
 // ---------------------------------------------------------------- prepare
-__global__ void __launch_bounds__(256)
-init_slots_kernel(const int32_t* __restrict__ cu_vis, int B, int32_t* __restrict__ assign,
-                  unsigned long long* __restrict__ best) {
-  const int g = blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= cu_vis[B]) return;
-  assign[g] = -1;
-  best[g] = 0ull;
-}
+// One block per visual row: its slot in the kept list (binary search of the ascending
+// list; -1 for a pruned row), a cleared arg-max word, the inverse norm, and, for kept
+// rows, a copy into the packed second operand of the similarity.
+constexpr int kPrepThreads = 128;
+constexpr int kPrepVec = 4;          // 16-byte vectors per thread and pass
 
-__global__ void __launch_bounds__(256)
-scatter_slots_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ cu_kept,
-                     const int32_t* __restrict__ cu_vis, int B, int32_t* __restrict__ assign) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= cu_kept[B]) return;
-  const int b = find_segment(cu_kept, B, i);
-  assign[cu_vis[b] + kept_idx[i]] = i - cu_kept[b];
-}
-
-// one block per visual row: inverse norm; kept rows are also copied to their slot
 template <typename T>
-__global__ void __launch_bounds__(128)
-rownorm_gather_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu_seqlens,
-                      const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ cu_kept,
-                      const int32_t* __restrict__ assign, int D, float* __restrict__ inv_norm,
-                      float* __restrict__ inv_norm_kept, T* __restrict__ kept_rows) {
+__global__ void __launch_bounds__(kPrepThreads)
+prepare_rows_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu_seqlens,
+                    const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ kept_idx,
+                    const int32_t* __restrict__ cu_kept, int D, int32_t* __restrict__ assign,
+                    unsigned long long* __restrict__ best, float* __restrict__ inv_norm,
+                    float* __restrict__ inv_norm_kept, T* __restrict__ kept_rows) {
   constexpr int kVec = Storage<T>::kVec;
   const int b = blockIdx.y, m = blockIdx.x;
   const int v0 = cu_vis[b];
   if (m >= cu_vis[b + 1] - v0) return;
   const int g = v0 + m;
-  const T* src = hidden + (size_t)(cu_seqlens[b] + m) * D;
-  const int slot = assign[g];
-  T* dst = slot >= 0 ? kept_rows + (size_t)(cu_kept[b] + slot) * D : nullptr;
-  float ss = 0.f;
-  for (int c = threadIdx.x * kVec; c < D; c += blockDim.x * kVec) {
-    float f[kVec];
-    Storage<T>::load(src + c, f);
-#pragma unroll
-    for (int i = 0; i < kVec; ++i) ss = fmaf(f[i], f[i], ss);
-    if (dst != nullptr) Storage<T>::store(dst + c, f);
+  const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
+  int lo = 0, hi = kb;                                   // first kept position >= m
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (kept_idx[k0 + mid] < m) lo = mid + 1; else hi = mid;
   }
-  __shared__ float red[4];
+  const int slot = (lo < kb && kept_idx[k0 + lo] == m) ? lo : -1;
+  const T* src = hidden + (size_t)(cu_seqlens[b] + m) * D;
+  T* dst = slot >= 0 ? kept_rows + (size_t)(k0 + slot) * D : nullptr;
+  float ss = 0.f;
+  for (int c0 = threadIdx.x * kVec; c0 < D; c0 += kPrepThreads * kVec * kPrepVec) {
+    float f[kPrepVec][kVec];
+#pragma unroll
+    for (int v = 0; v < kPrepVec; ++v) {                 // all loads of the pass are issued before any is used
+      const int c = c0 + v * kPrepThreads * kVec;
+      if (c < D) Storage<T>::load(src + c, f[v]);
+    }
+#pragma unroll
+    for (int v = 0; v < kPrepVec; ++v) {
+      const int c = c0 + v * kPrepThreads * kVec;
+      if (c < D) {
+#pragma unroll
+        for (int i = 0; i < kVec; ++i) ss = fmaf(f[v][i], f[v][i], ss);
+        if (dst != nullptr) Storage<T>::store(dst + c, f[v]);
+      }
+    }
+  }
+  __shared__ float red[kPrepThreads / 32];
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
@@ -65,7 +70,9 @@ rownorm_gather_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ 
     const float tot = (red[0] + red[1]) + (red[2] + red[3]);
     const float inv = tot > 0.f ? 1.0f / sqrtf(tot) : 0.f;
     inv_norm[g] = inv;
-    if (slot >= 0) inv_norm_kept[cu_kept[b] + slot] = inv;
+    assign[g] = slot;
+    best[g] = 0ull;
+    if (slot >= 0) inv_norm_kept[k0 + slot] = inv;
   }
 }
 
@@ -100,7 +107,7 @@ sim_simt_kernel(const T* __restrict__ hidden, const T* __restrict__ kept_rows,
       for (int i = 0; i < kVec; ++i) acc = fmaf(x[i], y[i], acc);
     }
     acc = warp_sum(acc);
-    const float sim = (acc * inm) * inv_norm_kept[k0 + s];   // the value the arg-max compares
+    const float sim = (acc * inm) * inv_norm_kept[k0 + s] + 0.0f;   // the value the arg-max compares (never -0)
     if (lane == 0) {
       const unsigned long long packed = ((unsigned long long)ordered_key(sim) << 32) | (0xffffffffu - (unsigned)s);
       mine = packed > mine ? packed : mine;
@@ -120,35 +127,40 @@ sim_simt_kernel(const T* __restrict__ hidden, const T* __restrict__ kept_rows,
 
 // ---------------------------------------------------------------- finish
 constexpr int kMemberThreads = 1024;
+constexpr int kMemberSmemSlots = 12 * 1024;        // kept counts up to this keep their counters in shared memory
 
 // One block per request: destination slots, member counts, list offsets and the
 // member lists (each list is put in ascending order by the aggregation kernel).
+// Counters live in shared memory when the kept count allows, else in `cursor`.
 __global__ void __launch_bounds__(kMemberThreads)
 members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ cu_kept,
                const unsigned long long* __restrict__ best, int32_t* __restrict__ assign,
                int32_t* __restrict__ member_count, int32_t* __restrict__ member_off,
                int32_t* __restrict__ cursor, int32_t* __restrict__ member_list) {
+  extern __shared__ int ctr_s[];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int v0 = cu_vis[b], V = cu_vis[b + 1] - v0;
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
   const int pruned_base = v0 - k0;                 // pruned tokens of earlier requests
+  int* ctr = kb <= kMemberSmemSlots ? ctr_s : cursor + k0;
   __shared__ int warp_tot[32];
   __shared__ int carry;
-  for (int s = tid; s < kb; s += kMemberThreads) cursor[k0 + s] = 0;
+  for (int s = tid; s < kb; s += kMemberThreads) ctr[s] = 0;
   __syncthreads();
   for (int m = tid; m < V; m += kMemberThreads) {
     const int g = v0 + m;
-    if (assign[g] < 0) {
-      const int slot = (int)(0xffffffffu - (unsigned)(best[g] & 0xffffffffull));
+    const unsigned long long w = best[g];
+    if (w != 0ull) {                               // a pruned token (kept tokens keep best == 0)
+      const int slot = (int)(0xffffffffu - (unsigned)(w & 0xffffffffull));
       assign[g] = slot;
-      atomicAdd(&cursor[k0 + slot], 1);
+      atomicAdd(&ctr[slot], 1);
     }
   }
   if (tid == 0) carry = 0;
   __syncthreads();
   for (int base = 0; base < kb; base += kMemberThreads) {
     const int s = base + tid;
-    const int c = s < kb ? cursor[k0 + s] : 0;
+    const int c = s < kb ? ctr[s] : 0;
     int incl = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -174,7 +186,7 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
     if (s < kb) {
       member_count[k0 + s] = c;
       member_off[k0 + s] = pruned_base + excl;
-      cursor[k0 + s] = pruned_base + excl;
+      ctr[s] = pruned_base + excl;
     }
     __syncthreads();
     if (tid == 0) carry += chunk_total;
@@ -182,62 +194,36 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
   }
   for (int m = tid; m < V; m += kMemberThreads) {
     const int g = v0 + m;
-    const int slot = assign[g];
-    // a kept token holds its own slot: tell it apart by asking whether it heads that slot
-    // (kept tokens were given their slot before this kernel and have best == 0)
-    if (best[g] != 0ull) member_list[atomicAdd(&cursor[k0 + slot], 1)] = m;
+    if (best[g] != 0ull) member_list[atomicAdd(&ctr[assign[g]], 1)] = m;
   }
 }
 
-constexpr int kAggThreads = 256;
-// kAggMaxVec: 16-byte vectors per thread, D <= 256 * kAggMaxVec * kVec
+__device__ __forceinline__ int ceil_div_dev(int a, int b) { return (a + b - 1) / b; }
 
-template <typename T, int kAggMaxVec>
-__device__ __forceinline__ void add_rows(const T* __restrict__ base, size_t row_stride, const int* list, int n,
-                                         int D, float (&acc)[kAggMaxVec][Storage<T>::kVec]) {
-  constexpr int kVec = Storage<T>::kVec;
-  int i = 0;
-  for (; i + 4 <= n; i += 4) {      // four rows in flight, added in list order
-    float f[4][kAggMaxVec][kVec];
+// acc += the 16 bytes of storage in `raw`, element by element
+template <typename T> __device__ __forceinline__ void add_raw(float (&acc)[Storage<T>::kVec], uint4 raw);
+template <> __device__ __forceinline__ void add_raw<float>(float (&acc)[4], uint4 raw) {
+  acc[0] += __uint_as_float(raw.x); acc[1] += __uint_as_float(raw.y);
+  acc[2] += __uint_as_float(raw.z); acc[3] += __uint_as_float(raw.w);
+}
+template <> __device__ __forceinline__ void add_raw<__nv_bfloat16>(float (&acc)[8], uint4 raw) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const T* src = base + (size_t)list[i + r] * row_stride;
-#pragma unroll
-      for (int v = 0; v < kAggMaxVec; ++v) {
-        const int c = (threadIdx.x + v * kAggThreads) * kVec;
-        if (c < D) Storage<T>::load(src + c, f[r][v]);
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int v = 0; v < kAggMaxVec; ++v) {
-        const int c = (threadIdx.x + v * kAggThreads) * kVec;
-        if (c < D) {
-#pragma unroll
-          for (int e = 0; e < kVec; ++e) acc[v][e] += f[r][v][e];
-        }
-      }
-  }
-  for (; i < n; ++i) {
-    const T* src = base + (size_t)list[i] * row_stride;
-#pragma unroll
-    for (int v = 0; v < kAggMaxVec; ++v) {
-      const int c = (threadIdx.x + v * kAggThreads) * kVec;
-      if (c < D) {
-        float f[kVec];
-        Storage<T>::load(src + c, f);
-#pragma unroll
-        for (int e = 0; e < kVec; ++e) acc[v][e] += f[e];
-      }
-    }
+  for (int i = 0; i < 4; ++i) {
+    acc[2 * i] += __uint_as_float(w[i] << 16);
+    acc[2 * i + 1] += __uint_as_float(w[i] & 0xffff0000u);
   }
 }
 
-// One block per OUTPUT row.  Rows [0, k_b) of a request are the merged kept
-// visual tokens, the rest are the prompt and response rows, copied.
-template <typename T, int kAggMaxVec>
-__global__ void __launch_bounds__(kAggThreads)
+constexpr int kAggMaxThreads = 512;
+constexpr int kAggUnroll = 8;            // member rows in flight per thread
+
+// One block per OUTPUT row, one 16-byte vector of the row per thread and pass.  Rows
+// [0, k_b) of a request are the merged kept visual tokens, the rest are the prompt and
+// response rows, copied.  Members are added in ascending position, kAggUnroll rows in
+// flight, fp32 accumulation, one rounding.
+template <typename T>
+__global__ void __launch_bounds__(kAggMaxThreads)
 aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu_seqlens,
                          const int32_t* __restrict__ n_visual, const int32_t* __restrict__ cu_vis,
                          const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ cu_kept,
@@ -253,12 +239,12 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
   const int lo = cu_seqlens[b], Vb = n_visual[b];
   T* dst = hidden_out + (size_t)row * D;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nwarps = nthreads >> 5;
 
   if (r >= kb) {                                    // prompt / response row: copy
     const int src_row = lo + Vb + (r - kb);
     const T* src = hidden + (size_t)src_row * D;
-    for (int c = tid * kVec; c < D; c += kAggThreads * kVec)
+    for (int c = tid * kVec; c < D; c += nthreads * kVec)
       *reinterpret_cast<uint4*>(dst + c) = *reinterpret_cast<const uint4*>(src + c);
     if (tid == 0) src_of_dst[row] = src_row;
     return;
@@ -266,65 +252,67 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
 
   const int pos = kept_idx[k0 + r];
   const int cnt = member_count[k0 + r];
+  const int off = member_off[k0 + r];
   const T* req = hidden + (size_t)lo * D;
-  float acc[kAggMaxVec][kVec];
-  {
-    const T* src = req + (size_t)pos * D;
-#pragma unroll
-    for (int v = 0; v < kAggMaxVec; ++v) {
-      const int c = (tid + v * kAggThreads) * kVec;
-      if (c < D) Storage<T>::load(src + c, acc[v]);
-      else {
-#pragma unroll
-        for (int e = 0; e < kVec; ++e) acc[v][e] = 0.f;
-      }
-    }
-  }
-  __shared__ int list[kAggThreads];
+  __shared__ int list[kAggMaxThreads];
+  __shared__ int warp_tot[kAggMaxThreads / 32];
+  const float inv_denom = mean ? 1.0f / (float)(1 + cnt) : 1.f;
   if (cnt > 0 && cnt <= 32) {
     // small list: rank-sort it inside one warp (members are distinct positions)
     if (warp == 0) {
-      const int mine = lane < cnt ? member_list[member_off[k0 + r] + lane] : 0x7fffffff;
+      const int mine = lane < cnt ? member_list[off + lane] : 0x7fffffff;
       int rank = 0;
       for (int j = 0; j < cnt; ++j) rank += __shfl_sync(0xffffffffu, mine, j) < mine ? 1 : 0;
       if (lane < cnt) list[rank] = mine;
     }
     __syncthreads();
-    add_rows<T, kAggMaxVec>(req, (size_t)D, list, cnt, D, acc);
-  } else if (cnt > 32) {
-    // long list: walk the request's assignment array in position order, 256
-    // positions at a time, compacting the members of this slot in order
-    __shared__ int warp_tot[kAggThreads / 32];
-    const int32_t* as = assign + cu_vis[b];
-    for (int base = 0; base < Vb; base += kAggThreads) {
-      const int m = base + tid;
-      // a member is a position routed to this slot that is not the kept token itself
-      const bool hit = m < Vb && as[m] == r && m != pos;
-      const unsigned bal = __ballot_sync(0xffffffffu, hit);
-      if (lane == 0) warp_tot[warp] = __popc(bal);
-      __syncthreads();
-      int before = 0, total = 0;
-#pragma unroll
-      for (int w = 0; w < kAggThreads / 32; ++w) {
-        const int t = warp_tot[w];
-        if (w < warp) before += t;
-        total += t;
-      }
-      if (hit) list[before + __popc(bal & ((1u << lane) - 1u))] = m;
-      __syncthreads();
-      add_rows<T, kAggMaxVec>(req, (size_t)D, list, total, D, acc);
-      __syncthreads();
-    }
   }
-  const float denom = mean ? (float)(1 + cnt) : 1.f;
+  const int passes = ceil_div_dev(D, nthreads * kVec);            // uniform over the block
+  for (int p = 0; p < passes; ++p) {
+    const int c = (p * nthreads + tid) * kVec;
+    const bool live = c < D;
+    const T* col = req + (live ? c : 0);                        // threads past the row end read column 0, write nothing
+    float acc[kVec];
+    Storage<T>::load(col + (size_t)pos * D, acc);
+    auto add_list = [&](int n) {
+      int i = 0;
+      for (; i + kAggUnroll <= n; i += kAggUnroll) {
+        uint4 raw[kAggUnroll];
 #pragma unroll
-  for (int v = 0; v < kAggMaxVec; ++v) {
-    const int c = (tid + v * kAggThreads) * kVec;
-    if (c < D) {
-      float f[kVec];
+        for (int u = 0; u < kAggUnroll; ++u) raw[u] = *reinterpret_cast<const uint4*>(col + (size_t)list[i + u] * D);
 #pragma unroll
-      for (int e = 0; e < kVec; ++e) f[e] = acc[v][e] / denom;
-      Storage<T>::store(dst + c, f);
+        for (int u = 0; u < kAggUnroll; ++u) add_raw<T>(acc, raw[u]);
+      }
+      for (; i < n; ++i) add_raw<T>(acc, *reinterpret_cast<const uint4*>(col + (size_t)list[i] * D));
+    };
+    if (cnt <= 32) {
+      add_list(cnt);
+    } else {
+      // long list: walk the request's assignment array in position order, one block-width of
+      // positions at a time, compacting the members of this slot in order
+      const int32_t* as = assign + cu_vis[b];
+      for (int base = 0; base < Vb; base += nthreads) {
+        const int m = base + tid;
+        const bool hit = m < Vb && as[m] == r && m != pos;     // routed here and not the kept token itself
+        const unsigned bal = __ballot_sync(0xffffffffu, hit);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int w = 0; w < nwarps; ++w) {
+          const int t = warp_tot[w];
+          if (w < warp) before += t;
+          total += t;
+        }
+        if (hit) list[before + __popc(bal & ((1u << lane) - 1u))] = m;
+        __syncthreads();
+        add_list(total);
+        __syncthreads();
+      }
+    }
+    if (live) {
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) acc[e] *= inv_denom;
+      Storage<T>::store(dst + c, acc);
     }
   }
   if (tid == 0) src_of_dst[row] = lo + pos;
@@ -333,22 +321,18 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
 }  // namespace
 
 int launch_merge_prepare(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
-  const int vis_bound = a.total_tokens < a.B * a.max_visual ? a.total_tokens : a.B * a.max_visual;
-  const int kept_bound = a.total_tokens < a.B * a.max_kept ? a.total_tokens : a.B * a.max_kept;
-  init_slots_kernel<<<ceil_div(vis_bound, 256), 256, 0, s>>>(a.cu_vis, a.B, a.assign, ctx->best);
-  D3TOM_LAUNCH_CHECK(ctx);
-  scatter_slots_kernel<<<ceil_div(kept_bound, 256), 256, 0, s>>>(a.kept_idx, a.cu_kept, a.cu_vis, a.B, a.assign);
-  D3TOM_LAUNCH_CHECK(ctx);
   dim3 grid(a.max_visual, a.B);
   if (a.dt == D3TOM_FP32)
-    rownorm_gather_kernel<float><<<grid, 128, 0, s>>>(static_cast<const float*>(a.hidden), a.cu_seqlens, a.cu_vis,
-                                                      a.cu_kept, a.assign, a.D, ctx->inv_norm, ctx->inv_norm_kept,
-                                                      static_cast<float*>(ctx->kept_rows));
+    prepare_rows_kernel<float><<<grid, kPrepThreads, 0, s>>>(static_cast<const float*>(a.hidden), a.cu_seqlens, a.cu_vis,
+                                                            a.kept_idx, a.cu_kept, a.D, a.assign, ctx->best,
+                                                            ctx->inv_norm, ctx->inv_norm_kept,
+                                                            static_cast<float*>(ctx->kept_rows));
   else
-    rownorm_gather_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(static_cast<const __nv_bfloat16*>(a.hidden),
-                                                              a.cu_seqlens, a.cu_vis, a.cu_kept, a.assign, a.D,
-                                                              ctx->inv_norm, ctx->inv_norm_kept,
-                                                              static_cast<__nv_bfloat16*>(ctx->kept_rows));
+    prepare_rows_kernel<__nv_bfloat16><<<grid, kPrepThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(a.hidden),
+                                                                    a.cu_seqlens, a.cu_vis, a.kept_idx, a.cu_kept, a.D,
+                                                                    a.assign, ctx->best, ctx->inv_norm,
+                                                                    ctx->inv_norm_kept,
+                                                                    static_cast<__nv_bfloat16*>(ctx->kept_rows));
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }
@@ -370,30 +354,31 @@ int launch_sim_simt(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
 }
 
 int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
-  members_kernel<<<a.B, kMemberThreads, 0, s>>>(a.cu_vis, a.cu_kept, ctx->best, a.assign, a.member_count,
-                                                ctx->member_off, ctx->member_cursor, ctx->member_list);
+  static bool attr_set = false;
+  if (!attr_set) {
+    D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(members_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kMemberSmemSlots * (int)sizeof(int)));
+    attr_set = true;
+  }
+  const size_t ctr_bytes = (size_t)(a.max_kept <= kMemberSmemSlots ? a.max_kept : 0) * sizeof(int);
+  members_kernel<<<a.B, kMemberThreads, ctr_bytes, s>>>(a.cu_vis, a.cu_kept, ctx->best, a.assign, a.member_count,
+                                                        ctx->member_off, ctx->member_cursor, ctx->member_list);
   D3TOM_LAUNCH_CHECK(ctx);
   const int mean = a.mode == D3TOM_AGG_MEAN ? 1 : 0;
   if (a.total_out <= 0) return D3TOM_OK;
-#define D3TOM_AGG_LAUNCH(T, NV)                                                                              \
-  aggregate_compact_kernel<T, NV><<<a.total_out, kAggThreads, 0, s>>>(                                       \
-      static_cast<const T*>(a.hidden), a.cu_seqlens, a.n_visual, a.cu_vis, a.kept_idx, a.cu_kept,            \
-      a.cu_seqlens_out, a.B, a.D, mean, a.assign, a.member_count, ctx->member_off, ctx->member_list,         \
-      static_cast<T*>(a.hidden_out), a.src_of_dst)
-  if (a.dt == D3TOM_FP32) {
-    const int nv = ceil_div(a.D, kAggThreads * 4);
-    if (nv <= 1) D3TOM_AGG_LAUNCH(float, 1);
-    else if (nv <= 2) D3TOM_AGG_LAUNCH(float, 2);
-    else if (nv <= 4) D3TOM_AGG_LAUNCH(float, 4);
-    else return D3TOM_ERR_UNSUPPORTED;
-  } else {
-    const int nv = ceil_div(a.D, kAggThreads * 8);
-    if (nv <= 1) D3TOM_AGG_LAUNCH(__nv_bfloat16, 1);
-    else if (nv <= 2) D3TOM_AGG_LAUNCH(__nv_bfloat16, 2);
-    else if (nv <= 4) D3TOM_AGG_LAUNCH(__nv_bfloat16, 4);
-    else return D3TOM_ERR_UNSUPPORTED;
-  }
-#undef D3TOM_AGG_LAUNCH
+  const int vec = a.dt == D3TOM_FP32 ? 4 : 8;
+  int threads = ceil_div(ceil_div(a.D, vec), 32) * 32;             // one 16-byte vector per thread when the row allows
+  if (threads > kAggMaxThreads) threads = kAggMaxThreads;
+  if (a.dt == D3TOM_FP32)
+    aggregate_compact_kernel<float><<<a.total_out, threads, 0, s>>>(
+        static_cast<const float*>(a.hidden), a.cu_seqlens, a.n_visual, a.cu_vis, a.kept_idx, a.cu_kept, a.cu_seqlens_out,
+        a.B, a.D, mean, a.assign, a.member_count, ctx->member_off, ctx->member_list, static_cast<float*>(a.hidden_out),
+        a.src_of_dst);
+  else
+    aggregate_compact_kernel<__nv_bfloat16><<<a.total_out, threads, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.n_visual, a.cu_vis, a.kept_idx, a.cu_kept,
+        a.cu_seqlens_out, a.B, a.D, mean, a.assign, a.member_count, ctx->member_off, ctx->member_list,
+        static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }
