@@ -29,7 +29,8 @@ void free_all(d3tom_ctx* c) {
   cudaFree(c->score_scratch); cudaFree(c->lse_scratch); cudaFree(c->imp_partial); cudaFree(c->imp_counters);
   cudaFree(c->inv_norm);
   cudaFree(c->inv_norm_kept); cudaFree(c->kept_rows); cudaFree(c->best); cudaFree(c->member_off);
-  cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->dev_status);
+  cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->heavy_slots); cudaFree(c->n_heavy);
+  cudaFree(c->dev_status);
 }
 
 bool dtype_ok(d3tom_dtype dt) { return dt == D3TOM_BF16 || dt == D3TOM_FP32; }
@@ -80,6 +81,8 @@ int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (st == D3TOM_OK) st = alloc(c, &c->member_off, T + 1);
   if (st == D3TOM_OK) st = alloc(c, &c->member_cursor, T);
   if (st == D3TOM_OK) st = alloc(c, &c->member_list, T);
+  if (st == D3TOM_OK) st = alloc(c, &c->heavy_slots, T / 32 + 1);
+  if (st == D3TOM_OK) st = alloc(c, &c->n_heavy, 1);
   if (st == D3TOM_OK) st = alloc(c, &c->dev_status, 1);
   if (st == D3TOM_OK && cudaMemset(c->dev_status, 0, sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st != D3TOM_OK) { free_all(c); delete c; return st; }

@@ -26,6 +26,8 @@ struct d3tom_ctx {
   int32_t* member_off;          // [max_total_tokens + 1] start of each kept slot's member list
   int32_t* member_cursor;       // [max_total_tokens]
   int32_t* member_list;         // [max_total_tokens] pruned positions grouped by destination slot
+  int32_t* heavy_slots;         // [max_total_tokens / 32 + 1] kept tokens with 32 members or more
+  int* n_heavy;                 // how many of them
   int* dev_status;              // device status word
   int vis_stride;               // row stride of score_scratch (floats)
 };

@@ -6,8 +6,8 @@
 //             every visual row, and a packed copy of the kept rows (the second
 //             operand of the similarity)
 //   sim_simt  cosine + arg-max on CUDA cores (fp32 storage, debugging aid)
-//   finish    destination slots, per-slot member lists, aggregation in
-//             ascending member order and compaction into the shortened sequence
+//   finish    destination slots, per-slot member lists, aggregation in a fixed
+//             order and compaction into the shortened sequence
 //
 // The arg-max is a 64-bit maximum over (order-preserving similarity bits << 32
 // | ~slot): the largest similarity wins and, among equals, the lowest slot, no
@@ -17,58 +17,90 @@
 namespace {
 
 // ---------------------------------------------------------------- prepare
-// One block per visual row: its slot in the kept list (binary search of the ascending
-// list; -1 for a pruned row), a cleared arg-max word, the inverse norm, and, for kept
-// rows, a copy into the packed second operand of the similarity.
-constexpr int kPrepThreads = 128;
-constexpr int kPrepVec = 4;          // 16-byte vectors per thread and pass
+// sum of squares of the 16 bytes of storage in `raw`
+template <typename T> __device__ __forceinline__ float sq_raw(uint4 raw);
+template <> __device__ __forceinline__ float sq_raw<float>(uint4 raw) {
+  const float a = __uint_as_float(raw.x), b = __uint_as_float(raw.y), c = __uint_as_float(raw.z), d = __uint_as_float(raw.w);
+  return fmaf(a, a, fmaf(b, b, fmaf(c, c, d * d)));
+}
+template <> __device__ __forceinline__ float sq_raw<__nv_bfloat16>(uint4 raw) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
+    s = fmaf(lo, lo, fmaf(hi, hi, s));
+  }
+  return s;
+}
+
+// One WARP per visual row (no block-wide synchronisation, so many rows are in flight per
+// SM): its slot in the kept list (-1 for a pruned row), a cleared arg-max word, the
+// inverse norm and, for kept rows, a copy into the packed second operand of the similarity.
+constexpr int kPrepWarps = 8;
+constexpr int kPrepInFlight = 8;       // 16-byte loads in flight per lane
 
 template <typename T>
-__global__ void __launch_bounds__(kPrepThreads)
+__global__ void __launch_bounds__(kPrepWarps * 32)
 prepare_rows_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu_seqlens,
                     const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ kept_idx,
                     const int32_t* __restrict__ cu_kept, int D, int32_t* __restrict__ assign,
                     unsigned long long* __restrict__ best, float* __restrict__ inv_norm,
                     float* __restrict__ inv_norm_kept, T* __restrict__ kept_rows) {
   constexpr int kVec = Storage<T>::kVec;
-  const int b = blockIdx.y, m = blockIdx.x;
+  const int b = blockIdx.y, lane = threadIdx.x & 31;
+  const int m = blockIdx.x * kPrepWarps + (threadIdx.x >> 5);
   const int v0 = cu_vis[b];
-  if (m >= cu_vis[b + 1] - v0) return;
+  if (m >= cu_vis[b + 1] - v0) return;                       // whole warp
   const int g = v0 + m;
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
-  int lo = 0, hi = kb;                                   // first kept position >= m
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if (kept_idx[k0 + mid] < m) lo = mid + 1; else hi = mid;
-  }
-  const int slot = (lo < kb && kept_idx[k0 + lo] == m) ? lo : -1;
-  const T* src = hidden + (size_t)(cu_seqlens[b] + m) * D;
-  T* dst = slot >= 0 ? kept_rows + (size_t)(k0 + slot) * D : nullptr;
-  float ss = 0.f;
-  for (int c0 = threadIdx.x * kVec; c0 < D; c0 += kPrepThreads * kVec * kPrepVec) {
-    float f[kPrepVec][kVec];
+  const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)(cu_seqlens[b] + m) * D);
+  const int n_vec = D / kVec;                                 // 16-byte vectors of the row
+  // the first batch of row loads goes out before the slot search so that the two latencies overlap
+  uint4 raw[kPrepInFlight];
 #pragma unroll
-    for (int v = 0; v < kPrepVec; ++v) {                 // all loads of the pass are issued before any is used
-      const int c = c0 + v * kPrepThreads * kVec;
-      if (c < D) Storage<T>::load(src + c, f[v]);
+  for (int u = 0; u < kPrepInFlight; ++u) {
+    const int vi = lane + u * 32;
+    if (vi < n_vec) raw[u] = src[vi];
+  }
+  // slot of position m in the ascending kept list: a 32-way search (each step narrows the range
+  // 32-fold with one load per lane and a ballot)
+  int lo = 0, len = kb;
+  while (len > 32) {
+    const int stride = (len + 31) >> 5;
+    const int idx = lo + lane * stride;
+    const bool le = idx < lo + len && kept_idx[k0 + idx] <= m;
+    const int n_le = __popc(__ballot_sync(0xffffffffu, le));   // lanes are ascending: the `le` lanes form a prefix
+    if (n_le == 0) { len = 0; break; }                          // every kept position is larger than m
+    const int new_lo = lo + (n_le - 1) * stride;
+    len = min(stride, lo + len - new_lo);
+    lo = new_lo;
+  }
+  const bool eq = lane < len && kept_idx[k0 + lo + lane] == m;
+  const unsigned eqb = __ballot_sync(0xffffffffu, eq);
+  const int slot = eqb ? lo + __ffs(eqb) - 1 : -1;
+  uint4* dst = slot >= 0 ? reinterpret_cast<uint4*>(kept_rows + (size_t)(k0 + slot) * D) : nullptr;
+  float ss = 0.f;
+  for (int base = 0; base < n_vec; base += kPrepInFlight * 32) {
+    if (base > 0) {
+#pragma unroll
+      for (int u = 0; u < kPrepInFlight; ++u) {
+        const int vi = base + lane + u * 32;
+        if (vi < n_vec) raw[u] = src[vi];
+      }
     }
 #pragma unroll
-    for (int v = 0; v < kPrepVec; ++v) {
-      const int c = c0 + v * kPrepThreads * kVec;
-      if (c < D) {
-#pragma unroll
-        for (int i = 0; i < kVec; ++i) ss = fmaf(f[v][i], f[v][i], ss);
-        if (dst != nullptr) Storage<T>::store(dst + c, f[v]);
+    for (int u = 0; u < kPrepInFlight; ++u) {
+      const int vi = base + lane + u * 32;
+      if (vi < n_vec) {
+        ss += sq_raw<T>(raw[u]);
+        if (dst != nullptr) dst[vi] = raw[u];
       }
     }
   }
-  __shared__ float red[kPrepThreads / 32];
   ss = warp_sum(ss);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const float tot = (red[0] + red[1]) + (red[2] + red[3]);
-    const float inv = tot > 0.f ? 1.0f / sqrtf(tot) : 0.f;
+  if (lane == 0) {
+    const float inv = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
     inv_norm[g] = inv;
     assign[g] = slot;
     best[g] = 0ull;
@@ -128,21 +160,28 @@ sim_simt_kernel(const T* __restrict__ hidden, const T* __restrict__ kept_rows,
 // ---------------------------------------------------------------- finish
 constexpr int kMemberThreads = 1024;
 constexpr int kMemberSmemSlots = 12 * 1024;        // kept counts up to this keep their counters in shared memory
+constexpr int kBitmapBytes = 64 * 1024;            // shared memory for the per-warp position bitmaps
+constexpr int kHeavy = 32;                         // a kept token with this many members or more is "heavy"
 
-// One block per request: destination slots, member counts, list offsets and the
-// member lists (each list is put in ascending order by the aggregation kernel).
-// Counters live in shared memory when the kept count allows, else in `cursor`.
+// One block per request: destination slots, member counts, list offsets and the member
+// lists.  Lists of fewer than kHeavy members are left in arrival order (the aggregation
+// kernel orders them inside a warp).  Heavy lists are rewritten in ascending position
+// here, by marking the members in a bitmap over the request's positions and reading the
+// bits back in order, and their slots are appended to `heavy_slots`.
+// Dynamic shared memory: [counters (kb ints, when kb <= kMemberSmemSlots)] [bitmaps].
 __global__ void __launch_bounds__(kMemberThreads)
 members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ cu_kept,
                const unsigned long long* __restrict__ best, int32_t* __restrict__ assign,
                int32_t* __restrict__ member_count, int32_t* __restrict__ member_off,
-               int32_t* __restrict__ cursor, int32_t* __restrict__ member_list) {
-  extern __shared__ int ctr_s[];
+               int32_t* __restrict__ cursor, int32_t* __restrict__ member_list,
+               int32_t* __restrict__ heavy_slots, int* __restrict__ n_heavy, int ctr_ints, int bitmap_warps) {
+  extern __shared__ int dyn_s[];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int v0 = cu_vis[b], V = cu_vis[b + 1] - v0;
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
   const int pruned_base = v0 - k0;                 // pruned tokens of earlier requests
-  int* ctr = kb <= kMemberSmemSlots ? ctr_s : cursor + k0;
+  int* ctr = kb <= ctr_ints ? dyn_s : cursor + k0;
+  unsigned* bitmaps = reinterpret_cast<unsigned*>(dyn_s + ctr_ints);
   __shared__ int warp_tot[32];
   __shared__ int carry;
   for (int s = tid; s < kb; s += kMemberThreads) ctr[s] = 0;
@@ -187,6 +226,7 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
       member_count[k0 + s] = c;
       member_off[k0 + s] = pruned_base + excl;
       ctr[s] = pruned_base + excl;
+      if (c >= kHeavy) heavy_slots[atomicAdd(n_heavy, 1)] = k0 + s;
     }
     __syncthreads();
     if (tid == 0) carry += chunk_total;
@@ -196,9 +236,44 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
     const int g = v0 + m;
     if (best[g] != 0ull) member_list[atomicAdd(&ctr[assign[g]], 1)] = m;
   }
+  __syncthreads();
+  // ---- heavy lists into ascending order (one warp per list, bitmap_warps warps take part)
+  if (warp < bitmap_warps) {
+    const int words = (V + 31) >> 5;
+    unsigned* bm = bitmaps + (size_t)warp * words;
+    for (int s = warp; s < kb; s += bitmap_warps) {
+      const int cnt = member_count[k0 + s];
+      if (cnt < kHeavy) continue;                  // uniform over the warp
+      const int off = member_off[k0 + s];
+      for (int w = lane; w < words; w += 32) bm[w] = 0u;
+      __syncwarp();
+      for (int i = lane; i < cnt; i += 32) {
+        const int m = member_list[off + i];
+        atomicOr(&bm[m >> 5], 1u << (m & 31));
+      }
+      __syncwarp();
+      int written = 0;
+      for (int w0 = 0; w0 < words; w0 += 32) {     // 32 words = 1024 positions per pass, in order
+        const int w = w0 + lane;
+        unsigned bits = w < words ? bm[w] : 0u;
+        const int n = __popc(bits);
+        int incl = n;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        int dst = off + written + incl - n;
+        while (bits) {
+          member_list[dst++] = (w << 5) + __ffs(bits) - 1;
+          bits &= bits - 1;
+        }
+        written += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      __syncwarp();
+    }
+  }
 }
-
-__device__ __forceinline__ int ceil_div_dev(int a, int b) { return (a + b - 1) / b; }
 
 // acc += the 16 bytes of storage in `raw`, element by element
 template <typename T> __device__ __forceinline__ void add_raw(float (&acc)[Storage<T>::kVec], uint4 raw);
@@ -215,124 +290,145 @@ template <> __device__ __forceinline__ void add_raw<__nv_bfloat16>(float (&acc)[
   }
 }
 
-constexpr int kAggMaxThreads = 512;
-constexpr int kAggUnroll = 8;            // member rows in flight per thread
+constexpr int kAggWarps = 8;
+constexpr int kAggUnroll = 4;            // rows in flight per lane
 
-// One block per OUTPUT row, one 16-byte vector of the row per thread and pass.  Rows
-// [0, k_b) of a request are the merged kept visual tokens, the rest are the prompt and
-// response rows, copied.  Members are added in ascending position, kAggUnroll rows in
-// flight, fp32 accumulation, one rounding.
+// acc += rows[0..n) of `req` (row indices held one per lane in `rows`), in that order,
+// kAggUnroll loads in flight
 template <typename T>
-__global__ void __launch_bounds__(kAggMaxThreads)
+__device__ __forceinline__ void add_rows(float (&acc)[Storage<T>::kVec], const T* req, int D, int rows, int n) {
+  for (int i = 0; i < n; i += kAggUnroll) {
+    uint4 raw[kAggUnroll];
+#pragma unroll
+    for (int u = 0; u < kAggUnroll; ++u) {
+      const int rr = __shfl_sync(0xffffffffu, rows, (i + u) & 31);
+      if (i + u < n) raw[u] = *reinterpret_cast<const uint4*>(req + (size_t)rr * D);
+    }
+#pragma unroll
+    for (int u = 0; u < kAggUnroll; ++u)
+      if (i + u < n) add_raw<T>(acc, raw[u]);
+  }
+}
+
+// Aggregation and compaction.  Blocks [0, light_blocks): one WARP per (output row, 512-byte
+// chunk of the row), one 16-byte vector per lane.  Rows [0, k_b) of a request are the
+// merged kept visual tokens, the rest are the prompt and response rows, copied.  The kept
+// row comes first, then its members in ascending position, fp32 accumulation, one rounding;
+// the (short) member list is ordered with shuffles inside the warp.
+// Blocks [light_blocks, ...): one BLOCK per (heavy kept token, chunk).  Its list is already
+// ascending; warp w adds the kept row (w = 0) and the 32-member segments w, w + 8, ...,
+// and the eight partial sums are added in warp order.  Every order is a fixed function of
+// the sorted list, so results do not depend on scheduling.
+template <typename T>
+__global__ void __launch_bounds__(kAggWarps * 32)
 aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu_seqlens,
-                         const int32_t* __restrict__ n_visual, const int32_t* __restrict__ cu_vis,
-                         const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ cu_kept,
-                         const int32_t* __restrict__ cu_seqlens_out, int B, int D, int mean,
-                         const int32_t* __restrict__ assign, const int32_t* __restrict__ member_count,
-                         const int32_t* __restrict__ member_off, const int32_t* __restrict__ member_list,
-                         T* __restrict__ hidden_out, int32_t* __restrict__ src_of_dst) {
+                         const int32_t* __restrict__ n_visual, const int32_t* __restrict__ kept_idx,
+                         const int32_t* __restrict__ cu_kept, const int32_t* __restrict__ cu_seqlens_out, int B, int D,
+                         int chunks, int total_out, int light_blocks, int mean,
+                         const int32_t* __restrict__ member_count, const int32_t* __restrict__ member_off,
+                         const int32_t* __restrict__ member_list, const int32_t* __restrict__ heavy_slots,
+                         const int* __restrict__ n_heavy, T* __restrict__ hidden_out, int32_t* __restrict__ src_of_dst) {
   constexpr int kVec = Storage<T>::kVec;
-  const int row = blockIdx.x;
-  if (row >= cu_seqlens_out[B]) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float acc[kVec];
+#pragma unroll
+  for (int e = 0; e < kVec; ++e) acc[e] = 0.f;
+
+  if ((int)blockIdx.x >= light_blocks) {
+    // ------------------------------------------------------------ a heavy kept token
+    const int item = (int)blockIdx.x - light_blocks;
+    const int hi = item / chunks, ch = item - hi * chunks;
+    if (hi >= *n_heavy) return;                                  // whole block
+    const int ks = heavy_slots[hi];                              // slot in the packed kept list
+    const int b = find_segment(cu_kept, B, ks);
+    const int r = ks - cu_kept[b];
+    const int lo = cu_seqlens[b];
+    const int row = cu_seqlens_out[b] + r;
+    const int c = (ch * 32 + lane) * kVec;
+    const bool live = c < D;
+    const T* req = hidden + (size_t)lo * D + (live ? c : 0);
+    const int pos = kept_idx[ks], cnt = member_count[ks], off = member_off[ks];
+    if (warp == 0) add_raw<T>(acc, *reinterpret_cast<const uint4*>(req + (size_t)pos * D));
+    for (int seg = warp; seg * 32 < cnt; seg += kAggWarps) {
+      const int n = min(32, cnt - seg * 32);
+      const int mine = lane < n ? member_list[off + seg * 32 + lane] : 0;
+      add_rows<T>(acc, req, D, mine, n);
+    }
+    __shared__ float part[kAggWarps][32][Storage<T>::kVec + 1];
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) part[warp][lane][e] = acc[e];
+    __syncthreads();
+    if (warp == 0 && live) {
+      for (int w = 1; w < kAggWarps; ++w)
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) acc[e] += part[w][lane][e];
+      const float inv_denom = mean ? 1.0f / (float)(1 + cnt) : 1.f;
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) acc[e] *= inv_denom;
+      Storage<T>::store(hidden_out + (size_t)row * D + c, acc);
+    }
+    if (ch == 0 && threadIdx.x == 0) src_of_dst[row] = lo + pos;
+    return;
+  }
+
+  const int gw = blockIdx.x * kAggWarps + warp;
+  const int row = gw / chunks, ch = gw - row * chunks;
+  if (row >= total_out) return;                                 // whole warp
   const int b = find_segment(cu_seqlens_out, B, row);
   const int r = row - cu_seqlens_out[b];
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
   const int lo = cu_seqlens[b], Vb = n_visual[b];
-  T* dst = hidden_out + (size_t)row * D;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nwarps = nthreads >> 5;
+  const int c = (ch * 32 + lane) * kVec;
+  const bool live = c < D;
+  const T* req = hidden + (size_t)lo * D + (live ? c : 0);      // lanes past the row end read column 0, write nothing
+  T* dst = hidden_out + (size_t)row * D + c;
 
-  if (r >= kb) {                                    // prompt / response row: copy
-    const int src_row = lo + Vb + (r - kb);
-    const T* src = hidden + (size_t)src_row * D;
-    for (int c = tid * kVec; c < D; c += nthreads * kVec)
-      *reinterpret_cast<uint4*>(dst + c) = *reinterpret_cast<const uint4*>(src + c);
-    if (tid == 0) src_of_dst[row] = src_row;
+  if (r >= kb) {                                                // prompt / response row: copy
+    const int src_row = Vb + (r - kb);
+    if (live) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(req + (size_t)src_row * D);
+    if (ch == 0 && lane == 0) src_of_dst[row] = lo + src_row;
     return;
   }
 
   const int pos = kept_idx[k0 + r];
   const int cnt = member_count[k0 + r];
   const int off = member_off[k0 + r];
-  const T* req = hidden + (size_t)lo * D;
-  __shared__ int list[kAggMaxThreads];
-  __shared__ int warp_tot[kAggMaxThreads / 32];
-  const float inv_denom = mean ? 1.0f / (float)(1 + cnt) : 1.f;
-  if (cnt > 0 && cnt <= 32) {
-    // small list: rank-sort it inside one warp (members are distinct positions)
-    if (warp == 0) {
-      const int mine = lane < cnt ? member_list[off + lane] : 0x7fffffff;
-      int rank = 0;
-      for (int j = 0; j < cnt; ++j) rank += __shfl_sync(0xffffffffu, mine, j) < mine ? 1 : 0;
-      if (lane < cnt) list[rank] = mine;
-    }
-    __syncthreads();
+  if (cnt >= kHeavy) return;                                    // a heavy block does this row
+  // lane t ends up holding the t-th row to add: the kept row, then the members by ascending
+  // position (distinct values, ranked by counting the smaller ones)
+  const int mine = lane < cnt ? member_list[off + lane] : 0x7fffffff;
+  int rank = 0;
+  for (int j = 0; j < cnt; ++j) rank += __shfl_sync(0xffffffffu, mine, j) < mine ? 1 : 0;
+  int ordered = pos;
+  for (int j = 0; j < cnt; ++j) {
+    const int v = __shfl_sync(0xffffffffu, mine, j), rj = __shfl_sync(0xffffffffu, rank, j);
+    if (lane == rj + 1) ordered = v;
   }
-  const int passes = ceil_div_dev(D, nthreads * kVec);            // uniform over the block
-  for (int p = 0; p < passes; ++p) {
-    const int c = (p * nthreads + tid) * kVec;
-    const bool live = c < D;
-    const T* col = req + (live ? c : 0);                        // threads past the row end read column 0, write nothing
-    float acc[kVec];
-    Storage<T>::load(col + (size_t)pos * D, acc);
-    auto add_list = [&](int n) {
-      int i = 0;
-      for (; i + kAggUnroll <= n; i += kAggUnroll) {
-        uint4 raw[kAggUnroll];
+  add_rows<T>(acc, req, D, ordered, cnt + 1);
+  if (live) {
+    const float inv_denom = mean ? 1.0f / (float)(1 + cnt) : 1.f;
 #pragma unroll
-        for (int u = 0; u < kAggUnroll; ++u) raw[u] = *reinterpret_cast<const uint4*>(col + (size_t)list[i + u] * D);
-#pragma unroll
-        for (int u = 0; u < kAggUnroll; ++u) add_raw<T>(acc, raw[u]);
-      }
-      for (; i < n; ++i) add_raw<T>(acc, *reinterpret_cast<const uint4*>(col + (size_t)list[i] * D));
-    };
-    if (cnt <= 32) {
-      add_list(cnt);
-    } else {
-      // long list: walk the request's assignment array in position order, one block-width of
-      // positions at a time, compacting the members of this slot in order
-      const int32_t* as = assign + cu_vis[b];
-      for (int base = 0; base < Vb; base += nthreads) {
-        const int m = base + tid;
-        const bool hit = m < Vb && as[m] == r && m != pos;     // routed here and not the kept token itself
-        const unsigned bal = __ballot_sync(0xffffffffu, hit);
-        if (lane == 0) warp_tot[warp] = __popc(bal);
-        __syncthreads();
-        int before = 0, total = 0;
-        for (int w = 0; w < nwarps; ++w) {
-          const int t = warp_tot[w];
-          if (w < warp) before += t;
-          total += t;
-        }
-        if (hit) list[before + __popc(bal & ((1u << lane) - 1u))] = m;
-        __syncthreads();
-        add_list(total);
-        __syncthreads();
-      }
-    }
-    if (live) {
-#pragma unroll
-      for (int e = 0; e < kVec; ++e) acc[e] *= inv_denom;
-      Storage<T>::store(dst + c, acc);
-    }
+    for (int e = 0; e < kVec; ++e) acc[e] *= inv_denom;
+    Storage<T>::store(dst, acc);
   }
-  if (tid == 0) src_of_dst[row] = lo + pos;
+  if (ch == 0 && lane == 0) src_of_dst[row] = lo + pos;
 }
 
 }  // namespace
 
 int launch_merge_prepare(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
-  dim3 grid(a.max_visual, a.B);
+  dim3 grid(ceil_div(a.max_visual, kPrepWarps), a.B);
   if (a.dt == D3TOM_FP32)
-    prepare_rows_kernel<float><<<grid, kPrepThreads, 0, s>>>(static_cast<const float*>(a.hidden), a.cu_seqlens, a.cu_vis,
-                                                            a.kept_idx, a.cu_kept, a.D, a.assign, ctx->best,
-                                                            ctx->inv_norm, ctx->inv_norm_kept,
-                                                            static_cast<float*>(ctx->kept_rows));
+    prepare_rows_kernel<float><<<grid, kPrepWarps * 32, 0, s>>>(static_cast<const float*>(a.hidden), a.cu_seqlens, a.cu_vis,
+                                                               a.kept_idx, a.cu_kept, a.D, a.assign, ctx->best,
+                                                               ctx->inv_norm, ctx->inv_norm_kept,
+                                                               static_cast<float*>(ctx->kept_rows));
   else
-    prepare_rows_kernel<__nv_bfloat16><<<grid, kPrepThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(a.hidden),
-                                                                    a.cu_seqlens, a.cu_vis, a.kept_idx, a.cu_kept, a.D,
-                                                                    a.assign, ctx->best, ctx->inv_norm,
-                                                                    ctx->inv_norm_kept,
-                                                                    static_cast<__nv_bfloat16*>(ctx->kept_rows));
+    prepare_rows_kernel<__nv_bfloat16><<<grid, kPrepWarps * 32, 0, s>>>(static_cast<const __nv_bfloat16*>(a.hidden),
+                                                                       a.cu_seqlens, a.cu_vis, a.kept_idx, a.cu_kept, a.D,
+                                                                       a.assign, ctx->best, ctx->inv_norm,
+                                                                       ctx->inv_norm_kept,
+                                                                       static_cast<__nv_bfloat16*>(ctx->kept_rows));
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }
@@ -357,28 +453,40 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   static bool attr_set = false;
   if (!attr_set) {
     D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(members_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kMemberSmemSlots * (int)sizeof(int)));
+                                             kMemberSmemSlots * (int)sizeof(int) + kBitmapBytes));
     attr_set = true;
   }
-  const size_t ctr_bytes = (size_t)(a.max_kept <= kMemberSmemSlots ? a.max_kept : 0) * sizeof(int);
-  members_kernel<<<a.B, kMemberThreads, ctr_bytes, s>>>(a.cu_vis, a.cu_kept, ctx->best, a.assign, a.member_count,
-                                                        ctx->member_off, ctx->member_cursor, ctx->member_list);
+  // shared memory of the members kernel: counters when they fit, then one position bitmap per sorting warp
+  const int ctr_ints = a.max_kept <= kMemberSmemSlots ? a.max_kept : 0;
+  const int words = ceil_div(a.max_visual > 0 ? a.max_visual : 1, 32);
+  int bitmap_warps = kBitmapBytes / (words * 4);
+  if (bitmap_warps > kMemberThreads / 32) bitmap_warps = kMemberThreads / 32;
+  if (bitmap_warps < 1) return D3TOM_ERR_UNSUPPORTED;              // more than 512 Ki visual tokens in one request
+  const size_t smem = (size_t)ctr_ints * sizeof(int) + (size_t)bitmap_warps * words * 4;
+  D3TOM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->n_heavy, 0, sizeof(int), s));
+  members_kernel<<<a.B, kMemberThreads, smem, s>>>(a.cu_vis, a.cu_kept, ctx->best, a.assign, a.member_count,
+                                                   ctx->member_off, ctx->member_cursor, ctx->member_list,
+                                                   ctx->heavy_slots, ctx->n_heavy, ctr_ints, bitmap_warps);
   D3TOM_LAUNCH_CHECK(ctx);
   const int mean = a.mode == D3TOM_AGG_MEAN ? 1 : 0;
   if (a.total_out <= 0) return D3TOM_OK;
   const int vec = a.dt == D3TOM_FP32 ? 4 : 8;
-  int threads = ceil_div(ceil_div(a.D, vec), 32) * 32;             // one 16-byte vector per thread when the row allows
-  if (threads > kAggMaxThreads) threads = kAggMaxThreads;
+  const int chunks = ceil_div(a.D, 32 * vec);                       // 512-byte chunks per row
+  const long long warps = (long long)a.total_out * chunks;
+  const int light_blocks = (int)((warps + kAggWarps - 1) / kAggWarps);
+  // at most (pruned tokens) / kHeavy kept tokens can be heavy; the blocks beyond the actual number leave at once
+  const int max_heavy = (a.total_tokens - a.total_out) / kHeavy;
+  const int blocks = light_blocks + max_heavy * chunks;
   if (a.dt == D3TOM_FP32)
-    aggregate_compact_kernel<float><<<a.total_out, threads, 0, s>>>(
-        static_cast<const float*>(a.hidden), a.cu_seqlens, a.n_visual, a.cu_vis, a.kept_idx, a.cu_kept, a.cu_seqlens_out,
-        a.B, a.D, mean, a.assign, a.member_count, ctx->member_off, ctx->member_list, static_cast<float*>(a.hidden_out),
-        a.src_of_dst);
+    aggregate_compact_kernel<float><<<blocks, kAggWarps * 32, 0, s>>>(
+        static_cast<const float*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out, a.B, a.D,
+        chunks, a.total_out, light_blocks, mean, a.member_count, ctx->member_off, ctx->member_list, ctx->heavy_slots,
+        ctx->n_heavy, static_cast<float*>(a.hidden_out), a.src_of_dst);
   else
-    aggregate_compact_kernel<__nv_bfloat16><<<a.total_out, threads, 0, s>>>(
-        static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.n_visual, a.cu_vis, a.kept_idx, a.cu_kept,
-        a.cu_seqlens_out, a.B, a.D, mean, a.assign, a.member_count, ctx->member_off, ctx->member_list,
-        static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
+    aggregate_compact_kernel<__nv_bfloat16><<<blocks, kAggWarps * 32, 0, s>>>(
+        static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out,
+        a.B, a.D, chunks, a.total_out, light_blocks, mean, a.member_count, ctx->member_off, ctx->member_list,
+        ctx->heavy_slots, ctx->n_heavy, static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }
