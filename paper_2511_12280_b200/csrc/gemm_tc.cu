@@ -8,22 +8,25 @@
 //             and folds every pruned row's candidates into its packed 64-bit
 //             running maximum, so the (V x k) similarity matrix never reaches HBM.
 //
-// One CTA computes a 128 x BN tile.  Warp 0 streams 128x64 / BNx64 operand tiles
-// with TMA into a ring of 128-byte-swizzled stages; one thread of warp 1 issues
-// tcgen05.mma (M = 128, N = BN, K = 16) into a TMEM accumulator; warps 2..5 read
-// the accumulator back with tcgen05.ld (one row per thread) and run the epilogue.
+// Persistent CTAs (one per SM) walk over the 128 x BN output tiles, M fastest so that the
+// BN x K operand stays hot in L2 while the M tiles that share it are computed.  Warps 0
+// and 6 stream 128x64 / BNx64 operand tiles with TMA into a ring of 128-byte-swizzled
+// stages and keep streaming across tile boundaries; one thread of warp 1 issues tcgen05.mma
+// (M = 128, N = BN, K = 16) into one of TWO TMEM accumulators; warps 2..5 read the other
+// accumulator back with tcgen05.ld (one row per thread) and run the epilogue meanwhile.
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace {
 
 constexpr int kBM = 128, kBK = 64;
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 224;      // warps: 0 A loads, 1 MMA, 2..5 epilogue, 6 B loads
 
 enum { kEpiProj = 0, kEpiSim = 1 };
 
 struct GemmParams {
   int num_k_blocks;           // K / 64
+  int m_tiles, n_tiles, batch;   // tile grid (per request for the similarity); tiles outside a request are skipped
   // projection
   __nv_bfloat16* out[3];      // q, k, v
   int out_rows;               // total tokens
@@ -36,9 +39,32 @@ struct GemmParams {
 };
 
 template <int BN> struct GemmSmem {
-  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kStages = BN == 256 ? 4 : (BN == 192 ? 5 : 6);   // as many as fit in 227 KB
+  static constexpr int kAccStride = BN <= 128 ? 128 : 256;              // TMEM columns between the two accumulators
   static constexpr int kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2;
   static constexpr int kBytes = kStages * (kABytes + kBBytes) + 1024 /*alignment slack*/ + 256 /*barriers*/ + BN * 4;
+};
+
+// Where tile `t` of the walk lies: rows of A, rows of B, and for the similarity the request
+// it belongs to.  Returns false for a tile of the bounding grid that a request does not reach.
+template <int BN, int EPI>
+struct TileCoord {
+  int m0, n0, a_row, b_row, b, Vb, kb, v0, k0;
+  __device__ __forceinline__ bool set(const GemmParams& p, int t) {
+    const int mi = t % p.m_tiles, rest = t / p.m_tiles;
+    const int ni = rest % p.n_tiles;
+    b = rest / p.n_tiles;
+    m0 = mi * kBM; n0 = ni * BN; a_row = m0; b_row = n0;
+    Vb = kb = v0 = k0 = 0;
+    if (EPI == kEpiSim) {
+      v0 = p.cu_vis[b]; Vb = p.cu_vis[b + 1] - v0;
+      k0 = p.cu_kept[b]; kb = p.cu_kept[b + 1] - k0;
+      if (m0 >= Vb || n0 >= kb || kb >= Vb) return false;   // nothing pruned in this request, or outside it
+      a_row = p.cu_seqlens[b] + m0;
+      b_row = k0 + n0;
+    }
+    return true;
+  }
 };
 
 template <int BN, int EPI>
@@ -52,91 +78,113 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* b_s = smem + kStages * S::kABytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * (S::kABytes + S::kBBytes));
   uint64_t* empty = full + kStages;
-  uint64_t* acc_full = empty + kStages;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+  uint64_t* acc_full = empty + kStages;       // [2]
+  uint64_t* acc_empty = acc_full + 2;         // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* ink_s = reinterpret_cast<float*>(smem + kStages * (S::kABytes + S::kBBytes) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN;
-
-  // tile coordinates in the operand matrices
-  int a_row = m0, b_row = n0;
-  int b = 0, Vb = 0, kb = 0, v0 = 0, k0 = 0;
-  if (EPI == kEpiSim) {
-    b = blockIdx.z;
-    v0 = p.cu_vis[b]; Vb = p.cu_vis[b + 1] - v0;
-    k0 = p.cu_kept[b]; kb = p.cu_kept[b + 1] - k0;
-    if (m0 >= Vb || n0 >= kb) return;          // uniform over the CTA, before any barrier or allocation
-    a_row = p.cu_seqlens[b] + m0;
-    b_row = k0 + n0;
-  }
+  const int total_tiles = p.m_tiles * p.n_tiles * p.batch;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
-    ptx::mbar_init(acc_full, 1);
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }   // A and B loaders
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }   // one arrival per epilogue warp
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
-  if (warp == 2) { ptx::tmem_alloc(tmem_slot, BN); ptx::tmem_relinquish(); }
-  if (EPI == kEpiSim) {
-    for (int j = threadIdx.x; j < BN; j += kGemmThreads) ink_s[j] = (n0 + j < kb) ? p.inv_norm_kept[k0 + n0 + j] : 0.f;
-  }
+  if (warp == 2) { ptx::tmem_alloc(tmem_slot, 2 * S::kAccStride); ptx::tmem_relinquish(); }
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
-  const uint32_t tmem_acc = *tmem_slot;
+  const uint32_t tmem_base = *tmem_slot;
+  TileCoord<BN, EPI> tc;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 6) {
+    // ------------------------------------------------------------ TMA producers: warp 0 streams A, warp 6 streams B
+    // (issuing a load and its barrier traffic costs the issuing thread a few hundred cycles per
+    // k-block; two threads keep ahead of 128 x 192 tiles, one does not)
     if (lane == 0) {
-      ptx::prefetch_tensormap(&tmap_a);
-      ptx::prefetch_tensormap(&tmap_b);
-      for (int kbk = 0; kbk < p.num_k_blocks; ++kbk) {
-        const int s = kbk % kStages;
-        if (!ptx::mbar_wait(&empty[s], ((kbk / kStages) & 1) ^ 1, abort_flag, p.dev_status)) break;
-        ptx::mbar_arrive_expect_tx(&full[s], S::kABytes + S::kBBytes);
-        ptx::tma_load_2d(a_s + s * S::kABytes, &tmap_a, &full[s], kbk * kBK, a_row);
-        ptx::tma_load_2d(b_s + s * S::kBBytes, &tmap_b, &full[s], kbk * kBK, b_row);
+      const bool is_a = warp == 0;
+      const CUtensorMap* tm = is_a ? &tmap_a : &tmap_b;
+      uint8_t* ring = is_a ? a_s : b_s;
+      const int stage_bytes = is_a ? S::kABytes : S::kBBytes;
+      ptx::prefetch_tensormap(tm);
+      int it = 0;                                   // k-blocks loaded so far, over all tiles
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        if (!tc.set(p, t)) continue;
+        const int row0 = is_a ? tc.a_row : tc.b_row;
+        for (int kbk = 0; kbk < p.num_k_blocks; ++kbk, ++it) {
+          const int s = it % kStages;
+          ok = ptx::mbar_wait(&empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.dev_status);
+          if (!ok) break;
+          ptx::mbar_arrive_expect_tx(&full[s], stage_bytes);
+          ptx::tma_load_2d(ring + s * stage_bytes, tm, &full[s], kbk * kBK, row0);
+        }
       }
     }
   } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, BN, 0, 0);
       const ptx::SmemDesc a_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(a_s));
       const ptx::SmemDesc b_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(b_s));
+      int it = 0, lt = 0;                           // k-blocks and tiles consumed so far
       bool ok = true;
-      for (int kbk = 0; kbk < p.num_k_blocks && ok; ++kbk) {
-        const int s = kbk % kStages;
-        ok = ptx::mbar_wait(&full[s], (kbk / kStages) & 1, abort_flag, p.dev_status);
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        if (!tc.set(p, t)) continue;
+        const int buf = lt & 1;
+        ok = ptx::mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1, abort_flag, p.dev_status);   // epilogue done with it
         if (!ok) break;
         ptx::tc_fence_after_sync();
-        const ptx::SmemDesc ad = ptx::smem_desc_advance(a_desc0, s * S::kABytes), bd = ptx::smem_desc_advance(b_desc0, s * S::kBBytes);
+        const uint32_t tmem_acc = tmem_base + (uint32_t)buf * S::kAccStride;
+        for (int kbk = 0; kbk < p.num_k_blocks; ++kbk, ++it) {
+          const int s = it % kStages;
+          ok = ptx::mbar_wait(&full[s], (it / kStages) & 1, abort_flag, p.dev_status);
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+          const ptx::SmemDesc ad = ptx::smem_desc_advance(a_desc0, s * S::kABytes), bd = ptx::smem_desc_advance(b_desc0, s * S::kBBytes);
 #pragma unroll
-        for (int kk = 0; kk < kBK / 16; ++kk) {
-          ptx::mma_ss(tmem_acc, ptx::smem_desc_advance(ad, kk * 32), ptx::smem_desc_advance(bd, kk * 32), idesc,
-                      (kbk > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < kBK / 16; ++kk) {
+            ptx::mma_ss(tmem_acc, ptx::smem_desc_advance(ad, kk * 32), ptx::smem_desc_advance(bd, kk * 32), idesc,
+                        (kbk > 0 || kk > 0) ? 1u : 0u);
+          }
+          ptx::mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
         }
-        ptx::mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
+        if (ok) ptx::mma_commit(&acc_full[buf]);
+        ++lt;
       }
-      if (ok) ptx::mma_commit(acc_full);
     }
   } else {
-    // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+    // ------------------------------------------------------------ epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;           // row of the tile owned by this thread
-    const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(acc_full, 0, abort_flag, p.dev_status));
-    ptx::tc_fence_after_sync();
-    if (ok) {
-      const uint32_t t_row = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+    const int et = threadIdx.x - 64;               // 0..127 among the epilogue threads
+    int lt = 0;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+      if (!tc.set(p, t)) continue;
+      const int buf = lt & 1;
+      if (EPI == kEpiSim) {
+        // inverse norms of this tile's kept rows; the four epilogue warps share them (named barrier 1)
+        asm volatile("bar.sync 1, 128;" ::: "memory");          // everyone is done with the previous tile's values
+        for (int j = et; j < BN; j += 128) ink_s[j] = (tc.n0 + j < tc.kb) ? p.inv_norm_kept[tc.k0 + tc.n0 + j] : 0.f;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[buf], (lt >> 1) & 1, abort_flag, p.dev_status));
+      if (!ok) break;
+      ptx::tc_fence_after_sync();
+      const uint32_t t_row = tmem_base + (uint32_t)buf * S::kAccStride + ((uint32_t)(quarter * 32) << 16);
       if (EPI == kEpiProj) {
-        const int grow = m0 + row;
-        const int which = n0 / p.out_cols, col0 = n0 % p.out_cols;   // BN divides D: a tile lies in one of q, k, v
-        __nv_bfloat16* dst = p.out[which] + (size_t)grow * p.out_cols + col0;
+        const int grow = tc.m0 + row;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           uint32_t r[32];
           ptx::tmem_ld32(t_row + c, r);
           ptx::tmem_wait_ld();
+          // 32 divides D, so a 32-column piece lies in one of q, k, v even when the tile straddles two of them
+          const int gcol = tc.n0 + c, which = gcol / p.out_cols;
+          __nv_bfloat16* dst = p.out[which] + (size_t)grow * p.out_cols + (gcol - which * p.out_cols) - c;
           if (grow < p.out_rows) {
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
@@ -151,13 +199,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       } else {
-        const int m = m0 + row;
-        const int g = v0 + m;
-        const bool active = m < Vb && p.assign[g] < 0;     // a pruned token of this request
+        const int m = tc.m0 + row;
+        const int g = tc.v0 + m;
+        const bool active = m < tc.Vb && p.assign[g] < 0;     // a pruned token of this request
         const float inm = active ? p.inv_norm[g] : 0.f;
         float best_sim = -INFINITY;                        // strict > below: the lowest slot wins a tie
         int best_slot = 0;
-        float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + n0 : nullptr;
+        float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + tc.n0 : nullptr;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           uint32_t r[32];
@@ -166,8 +214,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           if (active) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-              const int sidx = n0 + c + i;
-              if (sidx < kb) {
+              const int sidx = tc.n0 + c + i;
+              if (sidx < tc.kb) {
                 // the value the arg-max compares; + 0 turns a negative zero into the positive one
                 const float sim = (__uint_as_float(r[i]) * inm) * ink_s[c + i] + 0.0f;
                 if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
@@ -176,15 +224,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
           }
         }
-        const unsigned long long mine =
-            ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
-        if (active) atomicMax(p.best + g, mine);
+        if (active) {
+          const unsigned long long mine =
+              ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
+          atomicMax(p.best + g, mine);
+        }
       }
+      // the accumulator may be overwritten once all four warps have read it
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+      ++lt;
     }
     ptx::tc_fence_before_sync();
   }
   __syncthreads();
-  if (warp == 2) ptx::tmem_dealloc(tmem_acc, BN);
+  if (warp == 2) ptx::tmem_dealloc(tmem_base, 2 * S::kAccStride);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -204,7 +259,10 @@ EncodeTiledFn get_encode_fn() {
 }
 
 template <int BN, int EPI>
-int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, dim3 grid, cudaStream_t s) {
+int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t s) {
+  const long long tiles = (long long)p.m_tiles * p.n_tiles * p.batch;
+  if (tiles <= 0) return D3TOM_OK;
+  const int grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);          // persistent: one CTA per SM
   D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            GemmSmem<BN>::kBytes));
   gemm_tc_kernel<BN, EPI><<<grid, kGemmThreads, GemmSmem<BN>::kBytes, s>>>(ta, tb, p);
@@ -230,11 +288,7 @@ int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_
 
 int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int D, void* q, void* k, void* v,
                    cudaStream_t s) {
-  constexpr int BN = 256;
-  if (D % BN != 0) {
-    // narrow models: fall back to 128-wide tiles (D % 64 == 0 is checked by the caller)
-    if (D % 128 != 0) return D3TOM_ERR_UNSUPPORTED;
-  }
+  if (D % 128 != 0) return D3TOM_ERR_UNSUPPORTED;
   CUtensorMap ta, tb;
   int r = make_tmap_bf16_2d(&ta, x, (uint64_t)total, (uint64_t)D, (uint64_t)D, kBM);
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
@@ -242,14 +296,25 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
   p.num_k_blocks = D / kBK;
   p.out[0] = static_cast<__nv_bfloat16*>(q); p.out[1] = static_cast<__nv_bfloat16*>(k); p.out[2] = static_cast<__nv_bfloat16*>(v);
   p.out_rows = total; p.out_cols = D; p.dev_status = ctx->dev_status;
-  if (D % BN == 0) {
-    r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, BN);
-    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-    return launch_gemm<256, kEpiProj>(ctx, ta, tb, p, dim3(ceil_div(total, kBM), 3 * D / 256, 1), s);
+  p.m_tiles = ceil_div(total, kBM); p.batch = 1;
+  // Tile width: fewest (rounds of tiles over the SMs) x (measured cycles per 64-deep k-block at that
+  // width: 667 / 633 / 600 for 256 / 192 / 128 columns; narrow tiles pay the per-k-block barrier
+  // traffic of the issuing thread more often per unit of work).  192 divides 3 D whenever 64 divides D.
+  int bn = 128;
+  double best_cost = 1e30;
+  for (int cand : {256, 192, 128}) {
+    if ((3 * D) % cand != 0) continue;
+    const long long tiles = (long long)p.m_tiles * (3 * D / cand);
+    const double rounds = (double)((tiles + ctx->sm_count - 1) / ctx->sm_count);
+    const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
+    if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 128);
+  r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, (uint32_t)bn);
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-  return launch_gemm<128, kEpiProj>(ctx, ta, tb, p, dim3(ceil_div(total, kBM), 3 * D / 128, 1), s);
+  p.n_tiles = 3 * D / bn;
+  if (bn == 256) return launch_gemm<256, kEpiProj>(ctx, ta, tb, p, s);
+  if (bn == 192) return launch_gemm<192, kEpiProj>(ctx, ta, tb, p, s);
+  return launch_gemm<128, kEpiProj>(ctx, ta, tb, p, s);
 }
 
 int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
@@ -265,10 +330,13 @@ int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   p.cu_seqlens = a.cu_seqlens; p.cu_vis = a.cu_vis; p.cu_kept = a.cu_kept; p.assign = a.assign;
   p.inv_norm = ctx->inv_norm; p.inv_norm_kept = ctx->inv_norm_kept; p.best = ctx->best; p.sim_debug = a.sim_debug;
   p.max_kept = a.max_kept; p.dev_status = ctx->dev_status;
+  p.m_tiles = ceil_div(a.max_visual, kBM); p.batch = a.B;
   if (a.max_kept > 128) {      // 256-wide tiles: the A tile is streamed once per 256 kept rows and each MMA covers twice the work
     r = make_tmap_bf16_2d(&tb, ctx->kept_rows, (uint64_t)kept_rows_bound, (uint64_t)a.D, (uint64_t)a.D, 256);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-    return launch_gemm<256, kEpiSim>(ctx, ta, tb, p, dim3(ceil_div(a.max_visual, kBM), ceil_div(a.max_kept, 256), a.B), s);
+    p.n_tiles = ceil_div(a.max_kept, 256);
+    return launch_gemm<256, kEpiSim>(ctx, ta, tb, p, s);
   }
-  return launch_gemm<128, kEpiSim>(ctx, ta, tb, p, dim3(ceil_div(a.max_visual, kBM), ceil_div(a.max_kept, 128), a.B), s);
+  p.n_tiles = ceil_div(a.max_kept, 128);
+  return launch_gemm<128, kEpiSim>(ctx, ta, tb, p, s);
 }
