@@ -34,6 +34,8 @@ WORKLOAD_TEXT = {
     "C0": "C0: tiny fp32 merge layer, 256 visual + 16 prompt + 16 response tokens, 4 heads x 64, keep 0.25",
     "C1": "C1: LLaDA-8B-shaped merge layer, 1024 visual + 64 prompt + 64 response tokens, 32 heads x 128, keep 0.10",
     "C2": "C2: LLaDA-8B-shaped, 4096 visual + 128 prompt + 64 response tokens, 32 heads x 128, keep 0.25, 3 post-merge layers",
+    "C3": "C3: step schedule, 2048 visual + 64 prompt + 64 response tokens, 32 heads x 128, T = 64 denoising steps, "
+          "one more decider per step, keep ratio 0.5 -> 0 (mean 0.25), 3 post-merge layers; a step = one denoising step",
     "C4": "C4: 8 ragged requests, 1024-4096 visual tokens each, 32 heads x 128, keep in {0.1,0.25,0.5}, 3 post-merge layers",
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -120,7 +122,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ oracle timing
-def oracle_step_sample(w, heads=2, row_frac=8):
+def oracle_step_sample(w, heads=2, row_frac=8, decider_pos=None, keep=None):
     """Times the CPU oracle, as it stands, on a bounded sample of one step of
     workload ``w`` and extrapolates linearly to the full step:
     attention and importance on ``heads`` of the H heads (x H/heads), select and
@@ -132,19 +134,22 @@ def oracle_step_sample(w, heads=2, row_frac=8):
     hs = min(heads, H)
     scale = 1.0 / np.sqrt(dh)
     cu = w.cu_seqlens
-    q = w.q_for().to(dtype=__import__("torch").float64).numpy()
+    decider_pos = w.decider_pos if decider_pos is None else decider_pos
+    q = w.q_for(decider_pos).to(dtype=__import__("torch").float64).numpy()
     k = w.k.double().numpy()
     v = w.v.double().numpy()
-    dec = np.concatenate([np.asarray(d, np.int64) for d in w.decider_pos])
+    dec = np.concatenate([np.asarray(d, np.int64) for d in decider_pos])
     t = {}
     t0 = time.perf_counter()
     out_h = orc.attention(q[:, :hs], k[:, :hs], v[:, :hs], cu, scale)
     t["attn"] = (time.perf_counter() - t0) * H / hs
     t0 = time.perf_counter()
-    S = orc.importance(q[:, :hs], k[:, :hs], cu, w.n_visual, dec, w.cu_deciders(), scale)
+    S = orc.importance(q[:, :hs], k[:, :hs], cu, w.n_visual, dec, w.cu_deciders(decider_pos), scale)
     t["importance"] = (time.perf_counter() - t0) * H / hs
     t0 = time.perf_counter()
-    kept = [orc.select(S[b].astype(np.float32), orc.keep_count(w.n_visual[b], w.keep_ratio[b])) for b in range(w.B)]
+    if keep is None:
+        keep = [orc.keep_count(w.n_visual[b], w.keep_ratio[b]) for b in range(w.B)]
+    kept = [orc.select(S[b].astype(np.float32), keep[b]) for b in range(w.B)]
     t["select"] = time.perf_counter() - t0
     hidden = np.zeros((q.shape[0], H * dh))
     hidden[:, :hs * dh] = out_h
@@ -205,10 +210,18 @@ def main():
             return 0
         w = wl.config(args.config)
         config["requests_per_gpu"] = w.B
+        ref_kw = {}
+        if w.T:        # the schedule config is sampled at its middle step
+            from oracle import d3tom_oracle as orc
+            sm = w.T // 2
+            a_min = 2.0 * (1.0 - w.mean_keep_ratio) - 1.0
+            ref_kw = dict(decider_pos=w.step_deciders(sm),
+                          keep=[orc.keep_count(w.n_visual[0], 1.0 - orc.schedule_alpha(sm, w.T, a_min, 1.0))])
+            config["sampled_step"] = sm
         times = []
         desc, parts = "", {}
         for i in range(args.warmup + args.steps):
-            sec, desc, parts = oracle_step_sample(w)
+            sec, desc, parts = oracle_step_sample(w, **ref_kw)
             if i >= args.warmup:
                 times.append(sec)
         us = float(np.mean(times)) * 1e6
@@ -237,15 +250,33 @@ def main():
 
     w = wl.config(args.config)
     config["requests_per_gpu"] = w.B
-    keep = [B_.d3tom_keep_count(v, r) for v, r in zip(w.n_visual, w.keep_ratio)]
     total = int(w.cu_seqlens[-1])
-    step = MergeLayerStep(w.H, w.dh, w.torch_dtype, total, w.B, sum(len(d) for d in w.decider_pos), max(w.n_visual),
-                          n_post=len(w.w_post), mode=B_.AGG_MEAN, device=local_rank)
-    step.set_problem(w.n_visual, w.n_prompt, w.n_resp, w.decider_pos, keep)
-    q_h, k_h, v_h = (t.contiguous().pin_memory() for t in (w.q_for(), w.k, w.v))
-    q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
+    # one problem per schedule step (a single one for the constant-ratio configs)
+    if w.T:
+        a_min, a_max = 2.0 * (1.0 - w.mean_keep_ratio) - 1.0, 1.0
+        dec_steps = [w.step_deciders(s) for s in range(w.T)]
+        keep_steps = []
+        for s, dec in enumerate(dec_steps):
+            alpha = B_.d3tom_schedule_alpha(s, w.T, a_min, a_max)
+            # a step without deciders runs unmerged (Algorithm 1, else-branch)
+            keep_steps.append([B_.d3tom_keep_count(w.n_visual[0], 1.0 - alpha) if len(dec[0]) else w.n_visual[0]])
+        config["schedule"] = {"T": w.T, "alpha_min": a_min, "alpha_max": a_max, "keep_counts": [k[0] for k in keep_steps]}
+    else:
+        dec_steps = [w.decider_pos]
+        keep_steps = [[B_.d3tom_keep_count(v, r) for v, r in zip(w.n_visual, w.keep_ratio)]]
+    n_prob = len(dec_steps)
+    step = MergeLayerStep(w.H, w.dh, w.torch_dtype, total, w.B, max(sum(len(d) for d in dec) for dec in dec_steps),
+                          max(w.n_visual), n_post=len(w.w_post), mode=B_.AGG_MEAN, device=local_rank)
+    probs = [step.make_problem(w.n_visual, w.n_prompt, w.n_resp, dec, keep) for dec, keep in zip(dec_steps, keep_steps)]
+    step.use_problem(probs[n_prob // 2])
+    q_hs = [w.q_for(dec).contiguous().pin_memory() for dec in dec_steps]
+    k_h, v_h = w.k.contiguous().pin_memory(), w.v.contiguous().pin_memory()
+    qs = [t.to(dev) for t in q_hs]
+    q_h, q = q_hs[n_prob // 2], qs[n_prob // 2]
+    k, v = k_h.to(dev), v_h.to(dev)
+    q_stage = torch.empty_like(q)               # where the end-to-end path lands the step's Q
     w_post = [x.to(dev) for x in w.w_post]
-    out_h = torch.empty(step.total_out, step.D, dtype=w.torch_dtype).pin_memory()
+    out_h = torch.empty(total, step.D, dtype=w.torch_dtype).pin_memory()
 
     def sync_all():
         if world > 1:
@@ -264,7 +295,15 @@ def main():
     def max_over_ranks(x):
         return replicas.max_over_ranks(x, dev)
 
-    run = lambda: step.run(q, k, v, w_post)
+    counter = {"i": 0, "launches": 0}
+
+    def run():
+        i = counter["i"] % n_prob
+        counter["i"] += 1
+        step.use_problem(probs[i])
+        counter["launches"] += step.launches_per_step()
+        return step.run(qs[i], k, v, w_post)
+
     if args.only is not None:
         run()
         calls = {
@@ -290,7 +329,21 @@ def main():
     with ClockSampler(local_rank) as clk:
         clk.wait_started(run)          # keeps the GPU busy until the sampler delivers
         sync_all()
+        counter["launches"] = 0
         step_us = timed(run, args.steps)
+        launches_timed = counter["launches"]
+        sync_all()
+        # ---- per-step series of the schedule config: one event pair per denoising step, median of 3 trajectories
+        per_step = None
+        if w.T:
+            series = []
+            for _ in range(3):
+                counter["i"] = 0
+                series.append([timed(run, 1) for _ in range(n_prob)])
+            per_step = [float(x) for x in np.median(np.asarray(series), axis=0)]
+        # the breakdown below is taken at the middle problem
+        counter["i"] = n_prob // 2
+        run()
         sync_all()
         # ---- per-call breakdown (each call timed back to back on warm instruction caches;
         #      every call's working set is streamed from HBM or L2 as it would be inside the step)
@@ -313,15 +366,26 @@ def main():
     assert step.ctx.device_status() == 0, "device status word reports a kernel-side problem"
 
     # ---- end to end through the C ABI with host buffers: H2D of Q,K,V, the step, D2H of the result
+    e2e_bytes = {"h2d": 0, "d2h": 0, "n": 0}
+
     def e2e():
-        q.copy_(q_h, non_blocking=True); k.copy_(k_h, non_blocking=True); v.copy_(v_h, non_blocking=True)
-        y = step.run(q, k, v, w_post)
-        out_h.copy_(y[:step.total_out], non_blocking=True)
+        i = counter["i"] % n_prob
+        counter["i"] += 1
+        step.use_problem(probs[i])
+        q_stage.copy_(q_hs[i], non_blocking=True); k.copy_(k_h, non_blocking=True); v.copy_(v_h, non_blocking=True)
+        y = step.run(q_stage, k, v, w_post)
+        out_h[:step.total_out].copy_(y[:step.total_out], non_blocking=True)
+        e2e_bytes["h2d"] += 3 * q_stage.numel() * q_stage.element_size()
+        e2e_bytes["d2h"] += step.total_out * step.D * q_stage.element_size()
+        e2e_bytes["n"] += 1
     for _ in range(3):
         e2e()
     sync_all()
-    e2e_us = timed(e2e, min(50, max(5, args.steps // 2)))
+    counter["i"] = 0
+    e2e_bytes.update(h2d=0, d2h=0, n=0)
+    e2e_us = timed(e2e, max(n_prob, min(50, max(5, args.steps // 2))))
     sync_all()
+    step.use_problem(probs[n_prob // 2])
 
     step_us_max = max_over_ranks(step_us)
     e2e_us_max = max_over_ranks(e2e_us)
@@ -353,15 +417,22 @@ def main():
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
         "steps_per_s": world / (step_us_max * 1e-6),
         "e2e": {"value": e2e_us_max / world, "unit": "us",
-                "h2d_bytes_per_step": int(3 * q_h.numel() * q_h.element_size()),
-                "d2h_bytes_per_step": int(out_h.numel() * out_h.element_size())},
-        "gpu_launches": step.launches_per_step() * args.steps,
+                "h2d_bytes_per_step": int(e2e_bytes["h2d"] // max(1, e2e_bytes["n"])),
+                "d2h_bytes_per_step": int(e2e_bytes["d2h"] // max(1, e2e_bytes["n"]))},
+        "gpu_launches": int(launches_timed),
         "roofline": roofline, "breakdown_us": br, "derived": derived, "clocks": clocks,
         "peaks": dict(peaks, kind=peak_kind),
     }
 
+    if per_step is not None:
+        line["per_step_us"] = per_step
+        line["trajectory_total_us"] = float(sum(per_step))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sec, desc, parts = oracle_step_sample(w)
+        kw = {}
+        if w.T:
+            kw = dict(decider_pos=dec_steps[n_prob // 2], keep=keep_steps[n_prob // 2])
+            config["cpu_baseline_step"] = n_prob // 2
+        sec, desc, parts = oracle_step_sample(w, **kw)
         line["cpu_baseline"] = {"value": sec * 1e6, "unit": "us", "cores": blas_threads(), "kind": "oracle",
                                 "sample": desc, "breakdown_s": parts}
     if rank == 0:

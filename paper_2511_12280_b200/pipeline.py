@@ -11,6 +11,7 @@ between the calls.
 """
 from __future__ import annotations
 
+from types import SimpleNamespace
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -53,34 +54,44 @@ class MergeLayerStep:
         self.scale = 1.0 / float(np.sqrt(dh))
 
     # ------------------------------------------------------------------ problem description (small index arrays)
-    def set_problem(self, n_visual: Sequence[int], n_prompt: Sequence[int], n_resp: Sequence[int],
-                    decider_pos: List[np.ndarray], keep_count: Sequence[int]):
-        """Uploads the index arrays of a batch.  keep_count[b] = number of kept
-        visual tokens of request b (from d3tom_keep_count); a request without
-        deciders must be given keep_count = n_visual (Algorithm 1, else-branch)."""
-        self.nB = len(n_visual)
-        self.n_visual_h = [int(x) for x in n_visual]
-        self.seqlens_h = [int(v + p + o) for v, p, o in zip(n_visual, n_prompt, n_resp)]
-        self.keep_h = [int(x) for x in keep_count]
-        self.out_lens_h = [n - v + k for n, v, k in zip(self.seqlens_h, self.n_visual_h, self.keep_h)]
+    def make_problem(self, n_visual: Sequence[int], n_prompt: Sequence[int], n_resp: Sequence[int],
+                     decider_pos: List[np.ndarray], keep_count: Sequence[int]) -> SimpleNamespace:
+        """Uploads the index arrays of a batch and returns them with the host-side sizes the C ABI
+        wants.  keep_count[b] = number of kept visual tokens of request b (from d3tom_keep_count); a
+        request without deciders must be given keep_count = n_visual (Algorithm 1, else-branch).
+        Several problems can be prepared ahead (one per denoising step) and switched with
+        use_problem() without touching the device."""
+        pr = SimpleNamespace()
+        pr.nB = len(n_visual)
+        pr.n_visual_h = [int(x) for x in n_visual]
+        pr.seqlens_h = [int(v + p + o) for v, p, o in zip(n_visual, n_prompt, n_resp)]
+        pr.keep_h = [int(x) for x in keep_count]
+        pr.out_lens_h = [n - v + k for n, v, k in zip(pr.seqlens_h, pr.n_visual_h, pr.keep_h)]
         cs = lambda a: np.concatenate([[0], np.cumsum(a)]).astype(np.int32)
-        self.cu_seqlens_h, self.cu_vis_h = cs(self.seqlens_h), cs(self.n_visual_h)
-        self.cu_kept_h, self.cu_out_h = cs(self.keep_h), cs(self.out_lens_h)
-        self.cu_dec_h = cs([len(d) for d in decider_pos])
-        dec = np.concatenate([np.asarray(d, dtype=np.int32) for d in decider_pos]) if self.cu_dec_h[-1] else np.zeros(1, np.int32)
+        pr.cu_seqlens_h, pr.cu_vis_h = cs(pr.seqlens_h), cs(pr.n_visual_h)
+        pr.cu_kept_h, pr.cu_out_h = cs(pr.keep_h), cs(pr.out_lens_h)
+        pr.cu_dec_h = cs([len(d) for d in decider_pos])
+        dec = np.concatenate([np.asarray(d, dtype=np.int32) for d in decider_pos]) if pr.cu_dec_h[-1] else np.zeros(1, np.int32)
         d = self.dev
-        self.cu_seqlens, self.cu_vis = _i32(self.cu_seqlens_h, d), _i32(self.cu_vis_h, d)
-        self.cu_kept, self.cu_out = _i32(self.cu_kept_h, d), _i32(self.cu_out_h, d)
-        self.cu_dec, self.dec_pos = _i32(self.cu_dec_h, d), _i32(dec, d)
-        self.n_visual_d, self.keep_d = _i32(self.n_visual_h, d), _i32(self.keep_h, d)
-        self.total = int(self.cu_seqlens_h[-1])
-        self.total_vis = int(self.cu_vis_h[-1])
-        self.total_kept = int(self.cu_kept_h[-1])
-        self.total_out = int(self.cu_out_h[-1])
-        self.max_seqlen, self.max_visual = max(self.seqlens_h), max(self.n_visual_h)
-        self.max_kept, self.max_out = max(self.keep_h), max(self.out_lens_h)
+        pr.cu_seqlens, pr.cu_vis = _i32(pr.cu_seqlens_h, d), _i32(pr.cu_vis_h, d)
+        pr.cu_kept, pr.cu_out = _i32(pr.cu_kept_h, d), _i32(pr.cu_out_h, d)
+        pr.cu_dec, pr.dec_pos = _i32(pr.cu_dec_h, d), _i32(dec, d)
+        pr.n_visual_d, pr.keep_d = _i32(pr.n_visual_h, d), _i32(pr.keep_h, d)
+        pr.total = int(pr.cu_seqlens_h[-1])
+        pr.total_vis = int(pr.cu_vis_h[-1])
+        pr.total_kept = int(pr.cu_kept_h[-1])
+        pr.total_out = int(pr.cu_out_h[-1])
+        pr.max_seqlen, pr.max_visual = max(pr.seqlens_h), max(pr.n_visual_h)
+        pr.max_kept, pr.max_out = max(pr.keep_h), max(pr.out_lens_h)
+        return pr
+
+    def use_problem(self, pr: SimpleNamespace):
+        self.__dict__.update(vars(pr))
         if self.want_sim_debug:
-            self.sim_debug = torch.full((self.total_vis, self.max_kept), float("nan"), dtype=torch.float32, device=d)
+            self.sim_debug = torch.full((self.total_vis, self.max_kept), float("nan"), dtype=torch.float32, device=self.dev)
+
+    def set_problem(self, n_visual, n_prompt, n_resp, decider_pos, keep_count):
+        self.use_problem(self.make_problem(n_visual, n_prompt, n_resp, decider_pos, keep_count))
 
     # ------------------------------------------------------------------ the calls
     def attn_importance(self, q, k, v, stream=None):
@@ -117,7 +128,7 @@ class MergeLayerStep:
 
     def launches_per_step(self) -> int:
         """Kernels of this library launched by one run(): attention 1 + importance finish 1,
-        select 1, merge 3 (prepare) + 1 (similarity, when something is pruned) + 2 (finish),
-        and 2 per post-merge layer."""
+        select 1, merge 1 (prepare) + 1 (similarity, when something is pruned) + 2 (members,
+        aggregate/compact), and 2 per post-merge layer."""
         sim = 1 if self.total_out < self.total else 0
-        return 2 + 1 + 3 + sim + 2 + 2 * self.n_post
+        return 2 + 1 + 1 + sim + 2 + 2 * self.n_post
