@@ -38,6 +38,9 @@ WORKLOAD_TEXT = {
           "one more decider per step, keep ratio 0.5 -> 0 (mean 0.25), 3 post-merge layers; a step = one denoising step",
     "C4": "C4: 8 ragged requests, 1024-4096 visual tokens each, 32 heads x 128, keep in {0.1,0.25,0.5}, 3 post-merge layers",
 }
+# DRAM bytes of one launch of the dominant kernel from the committed ncu capture (null for configs not captured,
+# and to be reset to null whenever attn_tc.cu changes after the capture)
+ATTN_TRAFFIC_BYTES = {"C2": 164.3e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -396,7 +399,11 @@ def main():
     achieved = attn_flops / (attn_kernel_us * 1e-6) / 1e12
     roofline = {"bound": "tensor", "kernel": "attn_tc_kernel (merge-layer attention, timed alone)",
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_kind": peak_kind + " burst"}
+                "frac": achieved / peaks["bf16_tflops"], "traffic": ATTN_TRAFFIC_BYTES.get(args.config),
+                "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one merge-layer launch with the "
+                                "importance spill (profiles/attn_tc_kernel_c2_merge_layer.md); algorithmic bytes "
+                                "%.1f MB" % (4 * step.total * step.D * q.element_size() / 1e6),
+                "peak_kind": peak_kind + " burst"}
     merge_bytes = (step.total + step.total_out) * step.D * q.element_size()
     sim_flops = sum(2.0 * (v_ - k_) * k_ * step.D for v_, k_ in zip(step.n_visual_h, step.keep_h))
     post_attn_flops = sum(4.0 * n * n * step.D for n in step.out_lens_h)
