@@ -292,6 +292,7 @@ template <> __device__ __forceinline__ void add_raw<__nv_bfloat16>(float (&acc)[
 
 constexpr int kAggWarps = 8;
 constexpr int kAggUnroll = 4;            // rows in flight per lane
+constexpr int kAggCpw = 4;               // 512-byte chunks of a row handled by one warp of a light row
 
 // acc += rows[0..n) of `req` (row indices held one per lane in `rows`), in that order,
 // kAggUnroll loads in flight
@@ -310,8 +311,9 @@ __device__ __forceinline__ void add_rows(float (&acc)[Storage<T>::kVec], const T
   }
 }
 
-// Aggregation and compaction.  Blocks [0, light_blocks): one WARP per (output row, 512-byte
-// chunk of the row), one 16-byte vector per lane.  Rows [0, k_b) of a request are the
+// Aggregation and compaction.  Blocks [0, light_blocks): one WARP per (output row, group of
+// kAggCpw 512-byte chunks of the row), one 16-byte vector per lane and chunk, so that one chain
+// of index loads is followed by up to kAggUnroll x kAggCpw row loads in flight.  Rows [0, k_b) of a request are the
 // merged kept visual tokens, the rest are the prompt and response rows, copied.  The kept
 // row comes first, then its members in ascending position, fp32 accumulation, one rounding;
 // the (short) member list is ordered with shuffles inside the warp.
@@ -371,22 +373,34 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
     return;
   }
 
+  // ------------------------------------------------------------ light rows: one warp per (row, group of kAggCpw chunks)
+  const int groups = (chunks + kAggCpw - 1) / kAggCpw;
   const int gw = blockIdx.x * kAggWarps + warp;
-  const int row = gw / chunks, ch = gw - row * chunks;
+  const int row = gw / groups, cg = gw - row * groups;
   if (row >= total_out) return;                                 // whole warp
   const int b = find_segment(cu_seqlens_out, B, row);
   const int r = row - cu_seqlens_out[b];
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
   const int lo = cu_seqlens[b], Vb = n_visual[b];
-  const int c = (ch * 32 + lane) * kVec;
-  const bool live = c < D;
-  const T* req = hidden + (size_t)lo * D + (live ? c : 0);      // lanes past the row end read column 0, write nothing
-  T* dst = hidden_out + (size_t)row * D + c;
+  int col[kAggCpw];
+  bool live[kAggCpw];
+#pragma unroll
+  for (int j = 0; j < kAggCpw; ++j) {
+    col[j] = ((cg * kAggCpw + j) * 32 + lane) * kVec;
+    live[j] = col[j] < D;
+    if (!live[j]) col[j] = 0;                                   // lanes past the row end read column 0, write nothing
+  }
+  const T* req = hidden + (size_t)lo * D;
+  T* dst = hidden_out + (size_t)row * D;
 
   if (r >= kb) {                                                // prompt / response row: copy
     const int src_row = Vb + (r - kb);
-    if (live) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(req + (size_t)src_row * D);
-    if (ch == 0 && lane == 0) src_of_dst[row] = lo + src_row;
+    uint4 raw[kAggCpw];
+#pragma unroll
+    for (int j = 0; j < kAggCpw; ++j) raw[j] = *reinterpret_cast<const uint4*>(req + (size_t)src_row * D + col[j]);
+#pragma unroll
+    for (int j = 0; j < kAggCpw; ++j) if (live[j]) *reinterpret_cast<uint4*>(dst + col[j]) = raw[j];
+    if (cg == 0 && lane == 0) src_of_dst[row] = lo + src_row;
     return;
   }
 
@@ -404,14 +418,38 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
     const int v = __shfl_sync(0xffffffffu, mine, j), rj = __shfl_sync(0xffffffffu, rank, j);
     if (lane == rj + 1) ordered = v;
   }
-  add_rows<T>(acc, req, D, ordered, cnt + 1);
-  if (live) {
-    const float inv_denom = mean ? 1.0f / (float)(1 + cnt) : 1.f;
+  float accs[kAggCpw][kVec];
 #pragma unroll
-    for (int e = 0; e < kVec; ++e) acc[e] *= inv_denom;
-    Storage<T>::store(dst, acc);
+  for (int j = 0; j < kAggCpw; ++j)
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) accs[j][e] = 0.f;
+  const int n = cnt + 1;
+  for (int i = 0; i < n; i += kAggUnroll) {                     // kAggUnroll rows x kAggCpw chunks in flight
+    uint4 raw[kAggUnroll][kAggCpw];
+#pragma unroll
+    for (int u = 0; u < kAggUnroll; ++u) {
+      const int rr = __shfl_sync(0xffffffffu, ordered, (i + u) & 31);
+      if (i + u < n) {
+#pragma unroll
+        for (int j = 0; j < kAggCpw; ++j) raw[u][j] = *reinterpret_cast<const uint4*>(req + (size_t)rr * D + col[j]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kAggUnroll; ++u)
+      if (i + u < n) {
+#pragma unroll
+        for (int j = 0; j < kAggCpw; ++j) add_raw<T>(accs[j], raw[u][j]);
+      }
   }
-  if (ch == 0 && lane == 0) src_of_dst[row] = lo + pos;
+  const float inv_denom = mean ? 1.0f / (float)(1 + cnt) : 1.f;
+#pragma unroll
+  for (int j = 0; j < kAggCpw; ++j)
+    if (live[j]) {
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) accs[j][e] *= inv_denom;
+      Storage<T>::store(dst + col[j], accs[j]);
+    }
+  if (cg == 0 && lane == 0) src_of_dst[row] = lo + pos;
 }
 
 }  // namespace
@@ -472,7 +510,7 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   if (a.total_out <= 0) return D3TOM_OK;
   const int vec = a.dt == D3TOM_FP32 ? 4 : 8;
   const int chunks = ceil_div(a.D, 32 * vec);                       // 512-byte chunks per row
-  const long long warps = (long long)a.total_out * chunks;
+  const long long warps = (long long)a.total_out * ceil_div(chunks, kAggCpw);
   const int light_blocks = (int)((warps + kAggWarps - 1) / kAggWarps);
   // at most (pruned tokens) / kHeavy kept tokens can be heavy; the blocks beyond the actual number leave at once
   const int max_heavy = (a.total_tokens - a.total_out) / kHeavy;
