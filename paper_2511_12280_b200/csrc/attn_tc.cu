@@ -68,19 +68,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   constexpr int kTileBytes = S::kTileBytes;
   constexpr int kHalfBytes = kTile * 128;               // one 64-column sub-tile: 128 rows x 128 bytes
   constexpr int kHalves = DH / 64;
-  // CTAs of a request are dispatched in the order of their linear index (x fastest).  The first H
-  // indices take the LAST 256-row query block of every head: the response rows live there and
-  // decider rows do extra work, so those CTAs must not end up in the last wave.  The remaining
-  // indices walk head by head (one head's K/V stay hot in L2), query blocks from the end.
-  const int b = blockIdx.z;
-  const int linear = (int)blockIdx.y * (int)gridDim.x + (int)blockIdx.x, nqb = (int)gridDim.x;
+  // CTAs are dispatched in the order of their index.  Per request: the first H work items take the
+  // LAST 256-row query block of every head (the response rows live there and decider rows do extra
+  // work, so those CTAs must not end up in the last wave); the remaining items walk head by head
+  // (one head's K/V stay hot in L2), query blocks from the end.  Items from `split_from` on are cut
+  // into two CTAs of one 128-row tile each: the host does that to the items of an incomplete last
+  // wave, which then costs the time of a single tile instead of a pair.
+  const int items = a.H * a.nqb, per_req = items + (items - a.split_from);
+  const int b = (int)blockIdx.x / per_req, lin = (int)blockIdx.x - b * per_req;
+  int item = lin, half = -1;
+  if (lin >= a.split_from) { item = a.split_from + ((lin - a.split_from) >> 1); half = (lin - a.split_from) & 1; }
   int h, qb;
-  if (linear < a.H) { h = linear; qb = nqb - 1; }
-  else { const int r = linear - a.H; h = r / (nqb - 1); qb = nqb - 2 - r % (nqb - 1); }
+  if (item < a.H) { h = item; qb = a.nqb - 1; }
+  else { const int r = item - a.H; h = r / (a.nqb - 1); qb = a.nqb - 2 - r % (a.nqb - 1); }
   const int lo = a.cu_seqlens[b], n = a.cu_seqlens[b + 1] - lo;
-  const int q0 = qb * 2 * kTile;
+  const int q0 = qb * 2 * kTile + (half > 0 ? kTile : 0);
   if (q0 >= n) return;                                  // uniform; nothing allocated yet
-  const int n_qt = (n - q0 > kTile) ? 2 : 1;
+  const int n_qt = (half < 0 && n - q0 > kTile) ? 2 : 1;
   const int n_kv = (n + kTile - 1) / kTile;
 
   extern __shared__ uint8_t smem_raw[];
@@ -384,8 +388,17 @@ int launch(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
   D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            AttnSmem<DH>::kBytes));
-  dim3 grid(ceil_div(a.max_seqlen, 2 * kTile), a.H, a.B);
-  attn_tc_kernel<DH><<<grid, kAttnThreads, AttnSmem<DH>::kBytes, s>>>(tq, tk, tv, a);
+  AttnArgs k = a;
+  k.nqb = ceil_div(a.max_seqlen, 2 * kTile);
+  const int items = a.H * k.nqb, sms = ctx->sm_count;
+  k.split_from = items;
+  if (a.B == 1) {                                   // (with one request the row count is known here)
+    const int rest = items % sms;
+    if (2 * items <= sms) k.split_from = 0;                                   // tiny: single tiles reach more SMs
+    else if (items > sms && rest > 0 && 2 * rest <= sms) k.split_from = items - rest;   // incomplete last wave
+  }
+  const int grid = a.B * (items + (items - k.split_from));
+  attn_tc_kernel<DH><<<grid, kAttnThreads, AttnSmem<DH>::kBytes, s>>>(tq, tk, tv, k);
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }

@@ -122,6 +122,7 @@ struct AttnArgs {
   float scale_log2;             // softmax_scale * log2(e)
   float* score_scratch; float2* lse_scratch; int max_deciders; int vis_stride;
   int* dev_status;
+  int nqb, split_from;          // tensor-core kernel only, set by its launcher: 256-row blocks per request, first cut item
 };
 
 int launch_attn_simt(d3tom_ctx* ctx, d3tom_dtype dt, const AttnArgs& a, cudaStream_t s);
