@@ -30,7 +30,7 @@ void free_all(d3tom_ctx* c) {
   cudaFree(c->inv_norm);
   cudaFree(c->inv_norm_kept); cudaFree(c->kept_rows); cudaFree(c->best); cudaFree(c->member_off);
   cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->heavy_slots); cudaFree(c->n_heavy);
-  cudaFree(c->dev_status);
+  cudaFree(c->gemm_split_ws); cudaFree(c->gemm_split_counters); cudaFree(c->dev_status);
 }
 
 bool dtype_ok(d3tom_dtype dt) { return dt == D3TOM_BF16 || dt == D3TOM_FP32; }
@@ -83,6 +83,9 @@ int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (st == D3TOM_OK) st = alloc(c, &c->member_list, T);
   if (st == D3TOM_OK) st = alloc(c, &c->heavy_slots, T / 32 + 1);
   if (st == D3TOM_OK) st = alloc(c, &c->n_heavy, 1);
+  if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_ws, (size_t)2 * c->sm_count * 128 * 256);
+  if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_counters, (size_t)2 * c->sm_count);
+  if (st == D3TOM_OK && cudaMemset(c->gemm_split_counters, 0, 2 * c->sm_count * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st == D3TOM_OK) st = alloc(c, &c->dev_status, 1);
   if (st == D3TOM_OK && cudaMemset(c->dev_status, 0, sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st != D3TOM_OK) { free_all(c); delete c; return st; }

@@ -23,10 +23,14 @@ constexpr int kBM = 128, kBK = 64;
 constexpr int kGemmThreads = 224;      // warps: 0 A loads, 1 MMA, 2..5 epilogue, 6 B loads
 
 enum { kEpiProj = 0, kEpiSim = 1 };
+constexpr int kMaxKSplits = 4;        // K slices per similarity tile at most
 
 struct GemmParams {
   int num_k_blocks;           // K / 64
   int m_tiles, n_tiles, batch;   // tile grid (per request for the similarity); tiles outside a request are skipped
+  int k_splits;               // similarity with few tiles: each tile's K range is cut into this many work units
+  float* split_ws;            // [tiles * k_splits][BN][128] fp32 partial tiles (column-major: coalesced per warp)
+  int* split_counters;        // [tiles] parts done; zero between launches
   // projection
   __nv_bfloat16* out[3];      // q, k, v
   int out_rows;               // total tokens
@@ -85,7 +89,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   float* ink_s = reinterpret_cast<float*>(smem + kStages * (S::kABytes + S::kBBytes) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = p.m_tiles * p.n_tiles * p.batch;
+  const int total_units = p.m_tiles * p.n_tiles * p.batch * p.k_splits;   // a unit = one tile, or one K slice of a tile
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }   // A and B loaders
@@ -112,10 +116,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       ptx::prefetch_tensormap(tm);
       int it = 0;                                   // k-blocks loaded so far, over all tiles
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const int t = u / p.k_splits, sp = u - t * p.k_splits;
         if (!tc.set(p, t)) continue;
         const int row0 = is_a ? tc.a_row : tc.b_row;
-        for (int kbk = 0; kbk < p.num_k_blocks; ++kbk, ++it) {
+        const int kb0 = sp * p.num_k_blocks / p.k_splits, kb1 = (sp + 1) * p.num_k_blocks / p.k_splits;
+        for (int kbk = kb0; kbk < kb1; ++kbk, ++it) {
           const int s = it % kStages;
           ok = ptx::mbar_wait(&empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.dev_status);
           if (!ok) break;
@@ -132,14 +138,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const ptx::SmemDesc b_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(b_s));
       int it = 0, lt = 0;                           // k-blocks and tiles consumed so far
       bool ok = true;
-      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const int t = u / p.k_splits, sp = u - t * p.k_splits;
         if (!tc.set(p, t)) continue;
+        const int kb0 = sp * p.num_k_blocks / p.k_splits, kb1 = (sp + 1) * p.num_k_blocks / p.k_splits;
         const int buf = lt & 1;
         ok = ptx::mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1, abort_flag, p.dev_status);   // epilogue done with it
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t tmem_acc = tmem_base + (uint32_t)buf * S::kAccStride;
-        for (int kbk = 0; kbk < p.num_k_blocks; ++kbk, ++it) {
+        for (int kbk = kb0; kbk < kb1; ++kbk, ++it) {
           const int s = it % kStages;
           ok = ptx::mbar_wait(&full[s], (it / kStages) & 1, abort_flag, p.dev_status);
           if (!ok) break;
@@ -148,7 +156,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk) {
             ptx::mma_ss(tmem_acc, ptx::smem_desc_advance(ad, kk * 32), ptx::smem_desc_advance(bd, kk * 32), idesc,
-                        (kbk > 0 || kk > 0) ? 1u : 0u);
+                        (kbk > kb0 || kk > 0) ? 1u : 0u);
           }
           ptx::mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
         }
@@ -162,7 +170,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int row = quarter * 32 + lane;           // row of the tile owned by this thread
     const int et = threadIdx.x - 64;               // 0..127 among the epilogue threads
     int lt = 0;
-    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+    __shared__ int s_prev;
+    for (int u = blockIdx.x; u < total_units; u += gridDim.x) {
+      const int t = u / p.k_splits, sp = u - t * p.k_splits;
       if (!tc.set(p, t)) continue;
       const int buf = lt & 1;
       if (EPI == kEpiSim) {
@@ -199,36 +209,92 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       } else {
-        const int m = tc.m0 + row;
-        const int g = tc.v0 + m;
-        const bool active = m < tc.Vb && p.assign[g] < 0;     // a pruned token of this request
-        const float inm = active ? p.inv_norm[g] : 0.f;
-        float best_sim = -INFINITY;                        // strict > below: the lowest slot wins a tie
-        int best_slot = 0;
-        float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + tc.n0 : nullptr;
+        // With few tiles each tile's K range is cut into k_splits units on different SMs.  Every unit
+        // writes its partial sums out (column-major, so a warp's 32 rows are one 128-byte line); the
+        // unit that completes the tile (a counter, left at zero again) adds the parts in the order of
+        // the K slices and runs the arg-max on the sums: same values whichever unit comes last.
+        const bool split = p.k_splits > 1;
+        bool last = true;
+        if (split) {
+          float* part = p.split_ws + (size_t)(t * p.k_splits + sp) * BN * kBM;
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
-          uint32_t r[32];
-          ptx::tmem_ld32(t_row + c, r);
-          ptx::tmem_wait_ld();
-          if (active) {
+          for (int c = 0; c < BN; c += 32) {
+            uint32_t r[32];
+            ptx::tmem_ld32(t_row + c, r);
+            ptx::tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int sidx = tc.n0 + c + i;
-              if (sidx < tc.kb) {
-                // the value the arg-max compares; + 0 turns a negative zero into the positive one
-                const float sim = (__uint_as_float(r[i]) * inm) * ink_s[c + i] + 0.0f;
-                if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
-                if (dbg != nullptr) dbg[c + i] = sim;
+            for (int i = 0; i < 32; ++i) part[(size_t)(c + i) * kBM + row] = __uint_as_float(r[i]);
+          }
+          ptx::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);          // the accumulator is free again
+          __threadfence();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (et == 0) s_prev = atomicAdd(p.split_counters + t, 1);
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          last = s_prev == p.k_splits - 1;
+          if (last) {
+            if (et == 0) p.split_counters[t] = 0;
+            __threadfence();
+          }
+        }
+        if (last) {
+          const int m = tc.m0 + row;
+          const int g = tc.v0 + m;
+          const bool active = m < tc.Vb && p.assign[g] < 0;     // a pruned token of this request
+          const float inm = active ? p.inv_norm[g] : 0.f;
+          float best_sim = -INFINITY;                        // strict > below: the lowest slot wins a tie
+          int best_slot = 0;
+          float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + tc.n0 : nullptr;
+#pragma unroll 1
+          for (int c = 0; c < BN; c += 32) {
+            float dot[32];
+            if (!split) {
+              uint32_t r[32];
+              ptx::tmem_ld32(t_row + c, r);
+              ptx::tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) dot[i] = __uint_as_float(r[i]);
+            } else {
+              // all slices of the 32 columns are requested before any is added (one round trip, not k_splits)
+              float part[kMaxKSplits][32];
+#pragma unroll
+              for (int q = 0; q < kMaxKSplits; ++q) {
+                const float* src = p.split_ws + ((size_t)(t * p.k_splits + q) * BN + c) * kBM + row;
+                if (q < p.k_splits) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) part[q][i] = __ldcg(src + (size_t)i * kBM);
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < 32; ++i) dot[i] = 0.f;
+#pragma unroll
+              for (int q = 0; q < kMaxKSplits; ++q)
+                if (q < p.k_splits) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) dot[i] += part[q][i];
+                }
+            }
+            if (active) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                const int sidx = tc.n0 + c + i;
+                if (sidx < tc.kb) {
+                  // the value the arg-max compares; + 0 turns a negative zero into the positive one
+                  const float sim = (dot[i] * inm) * ink_s[c + i] + 0.0f;
+                  if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
+                  if (dbg != nullptr) dbg[c + i] = sim;
+                }
               }
             }
           }
+          if (active) {
+            const unsigned long long mine =
+                ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
+            atomicMax(p.best + g, mine);
+          }
         }
-        if (active) {
-          const unsigned long long mine =
-              ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
-          atomicMax(p.best + g, mine);
-        }
+        if (split) { ++lt; continue; }
       }
       // the accumulator may be overwritten once all four warps have read it
       ptx::tc_fence_before_sync();
@@ -260,7 +326,7 @@ EncodeTiledFn get_encode_fn() {
 
 template <int BN, int EPI>
 int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t s) {
-  const long long tiles = (long long)p.m_tiles * p.n_tiles * p.batch;
+  const long long tiles = (long long)p.m_tiles * p.n_tiles * p.batch * p.k_splits;
   if (tiles <= 0) return D3TOM_OK;
   const int grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);          // persistent: one CTA per SM
   D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -296,7 +362,7 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
   p.num_k_blocks = D / kBK;
   p.out[0] = static_cast<__nv_bfloat16*>(q); p.out[1] = static_cast<__nv_bfloat16*>(k); p.out[2] = static_cast<__nv_bfloat16*>(v);
   p.out_rows = total; p.out_cols = D; p.dev_status = ctx->dev_status;
-  p.m_tiles = ceil_div(total, kBM); p.batch = 1;
+  p.m_tiles = ceil_div(total, kBM); p.batch = 1; p.k_splits = 1;
   // Tile width: fewest (rounds of tiles over the SMs) x (measured cycles per 64-deep k-block at that
   // width: 667 / 633 / 600 for 256 / 192 / 128 columns; narrow tiles pay the per-k-block barrier
   // traffic of the issuing thread more often per unit of work).  192 divides 3 D whenever 64 divides D.
@@ -331,6 +397,18 @@ int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   p.inv_norm = ctx->inv_norm; p.inv_norm_kept = ctx->inv_norm_kept; p.best = ctx->best; p.sim_debug = a.sim_debug;
   p.max_kept = a.max_kept; p.dev_status = ctx->dev_status;
   p.m_tiles = ceil_div(a.max_visual, kBM); p.batch = a.B;
+  // Few tiles (short requests, small kept sets): a tile is 64 k-blocks of serial work on one SM while
+  // most SMs idle, so each tile's K range is cut into slices for different SMs (see the epilogue).
+  {
+    const int bn = a.max_kept > 128 ? 256 : 128;
+    const long long tiles = (long long)p.m_tiles * ceil_div(a.max_kept, bn) * p.batch;
+    int splits = (int)(ctx->sm_count / (tiles > 0 ? tiles : 1));
+    if (splits > kMaxKSplits) splits = kMaxKSplits;
+    if (splits > p.num_k_blocks) splits = p.num_k_blocks;
+    if (splits < 2 || tiles * splits > 2LL * ctx->sm_count) splits = 1;
+    p.k_splits = splits;
+    p.split_ws = ctx->gemm_split_ws; p.split_counters = ctx->gemm_split_counters;
+  }
   if (a.max_kept > 128) {      // 256-wide tiles: the A tile is streamed once per 256 kept rows and each MMA covers twice the work
     r = make_tmap_bf16_2d(&tb, ctx->kept_rows, (uint64_t)kept_rows_bound, (uint64_t)a.D, (uint64_t)a.D, 256);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }

@@ -311,13 +311,13 @@ __device__ __forceinline__ void add_rows(float (&acc)[Storage<T>::kVec], const T
   }
 }
 
-// Aggregation and compaction.  Blocks [0, light_blocks): one WARP per (output row, group of
+// Aggregation and compaction.  Blocks [heavy_blocks, ...): one WARP per (output row, group of
 // kAggCpw 512-byte chunks of the row), one 16-byte vector per lane and chunk, so that one chain
 // of index loads is followed by up to kAggUnroll x kAggCpw row loads in flight.  Rows [0, k_b) of a request are the
 // merged kept visual tokens, the rest are the prompt and response rows, copied.  The kept
 // row comes first, then its members in ascending position, fp32 accumulation, one rounding;
 // the (short) member list is ordered with shuffles inside the warp.
-// Blocks [light_blocks, ...): one BLOCK per (heavy kept token, chunk).  Its list is already
+// Blocks [0, heavy_blocks): one BLOCK per (heavy kept token, chunk); beyond the actual number they leave at once.  Its list is already
 // ascending; warp w adds the kept row (w = 0) and the 32-member segments w, w + 8, ...,
 // and the eight partial sums are added in warp order.  Every order is a fixed function of
 // the sorted list, so results do not depend on scheduling.
@@ -326,7 +326,7 @@ __global__ void __launch_bounds__(kAggWarps * 32)
 aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu_seqlens,
                          const int32_t* __restrict__ n_visual, const int32_t* __restrict__ kept_idx,
                          const int32_t* __restrict__ cu_kept, const int32_t* __restrict__ cu_seqlens_out, int B, int D,
-                         int chunks, int total_out, int light_blocks, int mean,
+                         int chunks, int total_out, int heavy_blocks, int mean,
                          const int32_t* __restrict__ member_count, const int32_t* __restrict__ member_off,
                          const int32_t* __restrict__ member_list, const int32_t* __restrict__ heavy_slots,
                          const int* __restrict__ n_heavy, T* __restrict__ hidden_out, int32_t* __restrict__ src_of_dst) {
@@ -336,9 +336,9 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
 #pragma unroll
   for (int e = 0; e < kVec; ++e) acc[e] = 0.f;
 
-  if ((int)blockIdx.x >= light_blocks) {
-    // ------------------------------------------------------------ a heavy kept token
-    const int item = (int)blockIdx.x - light_blocks;
+  if ((int)blockIdx.x < heavy_blocks) {
+    // ------------------------------------------------------------ a heavy kept token (these blocks take the longest: first in the grid)
+    const int item = (int)blockIdx.x;
     const int hi = item / chunks, ch = item - hi * chunks;
     if (hi >= *n_heavy) return;                                  // whole block
     const int ks = heavy_slots[hi];                              // slot in the packed kept list
@@ -375,7 +375,7 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
 
   // ------------------------------------------------------------ light rows: one warp per (row, group of kAggCpw chunks)
   const int groups = (chunks + kAggCpw - 1) / kAggCpw;
-  const int gw = blockIdx.x * kAggWarps + warp;
+  const int gw = ((int)blockIdx.x - heavy_blocks) * kAggWarps + warp;
   const int row = gw / groups, cg = gw - row * groups;
   if (row >= total_out) return;                                 // whole warp
   const int b = find_segment(cu_seqlens_out, B, row);
@@ -514,16 +514,17 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   const int light_blocks = (int)((warps + kAggWarps - 1) / kAggWarps);
   // at most (pruned tokens) / kHeavy kept tokens can be heavy; the blocks beyond the actual number leave at once
   const int max_heavy = (a.total_tokens - a.total_out) / kHeavy;
-  const int blocks = light_blocks + max_heavy * chunks;
+  const int heavy_blocks = max_heavy * chunks;
+  const int blocks = light_blocks + heavy_blocks;
   if (a.dt == D3TOM_FP32)
     aggregate_compact_kernel<float><<<blocks, kAggWarps * 32, 0, s>>>(
         static_cast<const float*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out, a.B, a.D,
-        chunks, a.total_out, light_blocks, mean, a.member_count, ctx->member_off, ctx->member_list, ctx->heavy_slots,
+        chunks, a.total_out, heavy_blocks, mean, a.member_count, ctx->member_off, ctx->member_list, ctx->heavy_slots,
         ctx->n_heavy, static_cast<float*>(a.hidden_out), a.src_of_dst);
   else
     aggregate_compact_kernel<__nv_bfloat16><<<blocks, kAggWarps * 32, 0, s>>>(
         static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out,
-        a.B, a.D, chunks, a.total_out, light_blocks, mean, a.member_count, ctx->member_off, ctx->member_list,
+        a.B, a.D, chunks, a.total_out, heavy_blocks, mean, a.member_count, ctx->member_off, ctx->member_list,
         ctx->heavy_slots, ctx->n_heavy, static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
