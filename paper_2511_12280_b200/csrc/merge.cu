@@ -338,9 +338,12 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
 
   if ((int)blockIdx.x < heavy_blocks) {
     // ------------------------------------------------------------ a heavy kept token (these blocks take the longest: first in the grid)
-    const int item = (int)blockIdx.x;
+    // (the host cannot know how many kept tokens are heavy: a fixed number of blocks walks over them)
+    const int n_items = *n_heavy * chunks;
+    for (int item = (int)blockIdx.x; item < n_items; item += heavy_blocks) {
     const int hi = item / chunks, ch = item - hi * chunks;
-    if (hi >= *n_heavy) return;                                  // whole block
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) acc[e] = 0.f;
     const int ks = heavy_slots[hi];                              // slot in the packed kept list
     const int b = find_segment(cu_kept, B, ks);
     const int r = ks - cu_kept[b];
@@ -370,6 +373,8 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
       Storage<T>::store(hidden_out + (size_t)row * D + c, acc);
     }
     if (ch == 0 && threadIdx.x == 0) src_of_dst[row] = lo + pos;
+    __syncthreads();                                            // `part` is reused by the next item
+    }
     return;
   }
 
@@ -514,7 +519,8 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   const int light_blocks = (int)((warps + kAggWarps - 1) / kAggWarps);
   // at most (pruned tokens) / kHeavy kept tokens can be heavy; the blocks beyond the actual number leave at once
   const int max_heavy = (a.total_tokens - a.total_out) / kHeavy;
-  const int heavy_blocks = max_heavy * chunks;
+  int heavy_blocks = max_heavy * chunks;
+  if (heavy_blocks > ctx->sm_count) heavy_blocks = ctx->sm_count;
   const int blocks = light_blocks + heavy_blocks;
   if (a.dt == D3TOM_FP32)
     aggregate_compact_kernel<float><<<blocks, kAggWarps * 32, 0, s>>>(
