@@ -188,6 +188,31 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
+def make_kv_cache_case(step, w, k, v, dev):
+    """Returns a callable that runs d3tom_merge_kv on the K/V rows of every request's [visual | prompt]
+    prefix with the kept set that the step's select produced."""
+    import torch
+    D = step.D
+    cu_full = step.cu_seqlens_h
+    rows = np.concatenate([np.arange(cu_full[b], cu_full[b] + w.n_visual[b] + w.n_prompt[b]) for b in range(w.B)])
+    idx = torch.as_tensor(rows, device=dev)
+    k_c, v_c = k.reshape(-1, D)[idx].contiguous(), v.reshape(-1, D)[idx].contiguous()
+    lens = [a + b for a, b in zip(w.n_visual, w.n_prompt)]
+    cs = lambda a: np.concatenate([[0], np.cumsum(a)]).astype(np.int32)
+    cu, cu_out = cs(lens), cs([n - vv + kk for n, vv, kk in zip(lens, w.n_visual, step.keep_h)])
+    t = lambda a: torch.as_tensor(np.asarray(a, np.int32), device=dev)
+    cu_d, cu_out_d = t(cu), t(cu_out)
+    total, total_out = int(cu[-1]), int(cu_out[-1])
+    k_o = torch.empty(total_out, D, dtype=k.dtype, device=dev); v_o = torch.empty_like(k_o)
+    assign = torch.empty(step.total_vis, dtype=torch.int32, device=dev)
+    mc = torch.empty(step.total_kept, dtype=torch.int32, device=dev)
+    src = torch.empty(total_out, dtype=torch.int32, device=dev)
+    nB, mode, ctx = step.nB, step.mode, step.ctx
+    nv, cv, ki, ck, mv, mk = step.n_visual_d, step.cu_vis, step.kept_idx, step.cu_kept, step.max_visual, step.max_kept
+    return lambda: ctx.d3tom_merge_kv(mode, k_c, v_c, cu_d, nv, cv, ki, ck, nB, D, total, total_out, mv, mk, k_o, v_o,
+                                      cu_out_d, assign, mc, src)
+
+
 # ------------------------------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -361,6 +386,9 @@ def main():
             br["attn_varlen"] = timed(lambda: step.ctx.d3tom_attn_varlen(step.q2, step.k2, step.v2, step.cu_out, step.nB,
                                                                         step.total_out, step.max_out, step.scale,
                                                                         step.layer_out[0]), reps)
+        # the same routing applied to the cached K/V prefix (Sec. 4.4): caches = K, V rows of [visual | prompt]
+        kv = make_kv_cache_case(step, w, k, v, dev)
+        br["merge_kv"] = timed(kv, reps)
         # the dominant kernel alone (no importance side-work): the attention kernel at the merge-layer length
         attn_kernel_us = timed(lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
                                                                   step.max_seqlen, step.scale, step.attn_out), reps)

@@ -10,6 +10,7 @@
  *   d3tom_merge             nearest-kept-neighbour routing by cosine similarity,
  *                           aggregation, physical removal of the merged rows
  *   d3tom_attn_varlen       bidirectional attention over the shortened sequences
+ *   d3tom_merge_kv          the same routing applied to a cached K/V prefix
  *   d3tom_proj_qkv          (supporting) Q,K,V projection of a post-merge layer
  *
  * Conventions shared by every call
@@ -211,6 +212,26 @@ int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode,
                 void* hidden_out, const int32_t* cu_seqlens_out,
                 int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
                 float* sim_debug, d3tom_stream stream);
+
+/* Sec. 4.4 (Compatibility with KV-Cache): the same merge applied to a cached prefix.
+ *
+ * k_cache, v_cache [total_tokens, D] hold, per request, the cached keys and values of its
+ * [visual | prompt] prefix (cu_seqlens gives the prefix lengths, n_visual the visual part).
+ * With the kept set K from d3tom_select and its complement M: every m in M is routed to
+ * pi(m) = argmax over k in K of cos(K_m, K_k) (full-width rows, pre-merge values, ties to
+ * the lowest kept position); then K_pi(m) += K_m and V_pi(m) += V_m (SUM, the paper's
+ * equations; MEAN divides both by 1 + members, one reading of "renormalise"), and the
+ * positions in M are dropped: k_out, v_out [total_out, D] are the shorter caches, rows
+ * ordered as in d3tom_merge.  Every other argument is as in d3tom_merge; assign,
+ * member_count and src_of_dst describe the routing shared by both tensors. */
+int d3tom_merge_kv(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode,
+                   const void* k_cache, const void* v_cache,
+                   const int32_t* cu_seqlens, const int32_t* n_visual, const int32_t* cu_vis,
+                   const int32_t* kept_idx, const int32_t* cu_kept,
+                   int B, int D, int total_tokens, int total_out, int max_visual, int max_kept,
+                   void* k_out, void* v_out, const int32_t* cu_seqlens_out,
+                   int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
+                   float* sim_debug, d3tom_stream stream);
 
 /* Sec. 3.2.2, last paragraph: the layers after l* run on the shortened tensor.
  * Same attention as d3tom_attn_importance, over packed ragged sequences, with

@@ -269,6 +269,43 @@ def merge(hidden, cu_seqlens, n_visual, kept_idx_list, mode=SUM, dtype="bf16", a
 
 
 # --------------------------------------------------------------------------
+# Sec. 4.4, compatibility with KV-cache: route by cosine on K, add K and V, drop
+# --------------------------------------------------------------------------
+def merge_kv(k_cache, v_cache, cu_seqlens, n_visual, kept_idx_list, mode=SUM, dtype="bf16", assignment_list=None):
+    """The merge applied to a cached [visual | prompt] prefix.  k_cache, v_cache:
+    [total, D] (storage precision); per request the kept set K = kept_idx_list[b]
+    and its complement M.  For every m in M, pi(m) = argmax_{k in K} cos(K_m, K_k)
+    on the pre-merge keys (first maximiser); K_pi(m) += K_m and V_pi(m) += V_m
+    (MEAN: both divided by 1 + members, the reading of "renormalise"); the
+    positions in M are dropped.  Returns dict with k_out, v_out, cu_seqlens_out,
+    src_of_dst, assign, member_count."""
+    k_cache = np.asarray(k_cache, np.float64)
+    v_cache = np.asarray(v_cache, np.float64)
+    k_outs, v_outs, srcs, assigns, counts = [], [], [], [], []
+    cu_out = [0]
+    for b in range(len(cu_seqlens) - 1):
+        lo, hi = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        Vb = int(n_visual[b])
+        kept = np.asarray(kept_idx_list[b], dtype=np.int64)
+        K, Vv = k_cache[lo:hi], v_cache[lo:hi]
+        pi = assign(K[:Vb], kept) if assignment_list is None else np.asarray(assignment_list[b])   # routing from the keys only
+        k_merged, cnt = aggregate(K[:Vb], kept, pi, mode)
+        v_merged, cnt_v = aggregate(Vv[:Vb], kept, pi, mode)
+        assert np.array_equal(cnt, cnt_v)
+        ko, src = compact(K, Vb, kept, round_storage(k_merged, dtype))
+        vo, _ = compact(Vv, Vb, kept, round_storage(v_merged, dtype))
+        k_outs.append(ko); v_outs.append(vo); srcs.append(src + lo); assigns.append(pi); counts.append(cnt)
+        cu_out.append(cu_out[-1] + ko.shape[0])
+    return {
+        "k_out": np.concatenate(k_outs, axis=0), "v_out": np.concatenate(v_outs, axis=0),
+        "cu_seqlens_out": np.asarray(cu_out, dtype=np.int32),
+        "src_of_dst": np.concatenate(srcs).astype(np.int32),
+        "assign": np.concatenate(assigns).astype(np.int32),
+        "member_count": np.concatenate(counts).astype(np.int32),
+    }
+
+
+# --------------------------------------------------------------------------
 # layers after l*: attention over the shortened sequence (Sec. 3.2.2, last
 # paragraph).  A "layer" here is attention only: X <- MHA(X; W_q, W_k, W_v).
 # --------------------------------------------------------------------------

@@ -52,6 +52,7 @@ _SIGNATURES = {
                                           _P]),
     "d3tom_select": (_I, [_P, _P, _P, _P, _P, _I, _I, _P, _P, _P]),
     "d3tom_merge": (_I, [_P, _I, _I, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P]),
+    "d3tom_merge_kv": (_I, [_P, _I, _I, _P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "d3tom_attn_varlen": (_I, [_P, _I, _P, _P, _P, _P, _I, _I, _I, _F, _P, _P]),
     "d3tom_proj_qkv": (_I, [_P, _I, _P, _P, _I, _I, _P, _P, _P, _P]),
 }
@@ -183,6 +184,15 @@ class Context:
                                   max_visual, max_kept, _ptr(hidden_out), _ptr(cu_seqlens_out), _ptr(assign),
                                   _ptr(member_count), _ptr(src_of_dst), _ptr(sim_debug), _stream(stream)),
                "d3tom_merge")
+
+    def d3tom_merge_kv(self, mode, k_cache, v_cache, cu_seqlens, n_visual, cu_vis, kept_idx, cu_kept, B, D, total_tokens,
+                       total_out, max_visual, max_kept, k_out, v_out, cu_seqlens_out, assign, member_count, src_of_dst,
+                       sim_debug=None, stream=None):
+        _check(load().d3tom_merge_kv(self._h, _dt(k_cache), mode, _ptr(k_cache), _ptr(v_cache), _ptr(cu_seqlens),
+                                     _ptr(n_visual), _ptr(cu_vis), _ptr(kept_idx), _ptr(cu_kept), B, D, total_tokens,
+                                     total_out, max_visual, max_kept, _ptr(k_out), _ptr(v_out), _ptr(cu_seqlens_out),
+                                     _ptr(assign), _ptr(member_count), _ptr(src_of_dst), _ptr(sim_debug),
+                                     _stream(stream)), "d3tom_merge_kv")
 
     def d3tom_attn_varlen(self, q, k, v, cu_seqlens, B, total_tokens, max_seqlen, softmax_scale, out, stream=None):
         _check(load().d3tom_attn_varlen(self._h, _dt(q), _ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), B,

@@ -226,17 +226,18 @@ int d3tom_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis,
                        static_cast<cudaStream_t>(stream));
 }
 
-int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* hidden, const int32_t* cu_seqlens,
-                const int32_t* n_visual, const int32_t* cu_vis, const int32_t* kept_idx, const int32_t* cu_kept,
-                int B, int D, int total_tokens, int total_out, int max_visual, int max_kept, void* hidden_out,
-                const int32_t* cu_seqlens_out, int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
-                float* sim_debug, d3tom_stream stream) {
+static int merge_common(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* hidden, const void* second,
+                        const int32_t* cu_seqlens, const int32_t* n_visual, const int32_t* cu_vis,
+                        const int32_t* kept_idx, const int32_t* cu_kept, int B, int D, int total_tokens, int total_out,
+                        int max_visual, int max_kept, void* hidden_out, void* second_out,
+                        const int32_t* cu_seqlens_out, int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
+                        float* sim_debug, cudaStream_t s) {
   if (ctx == nullptr) return D3TOM_ERR_INVALID_ARG;
   if (!dtype_ok(dt)) return D3TOM_ERR_UNSUPPORTED;
   if (mode != D3TOM_AGG_SUM && mode != D3TOM_AGG_MEAN) return D3TOM_ERR_INVALID_ARG;
   if (hidden == nullptr || cu_seqlens == nullptr || n_visual == nullptr || cu_vis == nullptr || kept_idx == nullptr ||
       cu_kept == nullptr || hidden_out == nullptr || cu_seqlens_out == nullptr || assign == nullptr ||
-      member_count == nullptr || src_of_dst == nullptr)
+      member_count == nullptr || src_of_dst == nullptr || (second == nullptr) != (second_out == nullptr))
     return D3TOM_ERR_INVALID_ARG;
   if (B <= 0 || D <= 0 || total_tokens < 0 || total_out < 0 || total_out > total_tokens || max_visual < 0 ||
       max_kept < 0 || max_kept > max_visual || max_visual > total_tokens)
@@ -247,7 +248,6 @@ int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* hidd
   if (total_tokens == 0) return D3TOM_OK;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return D3TOM_ERR_CUDA;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   MergeArgs a;
   a.dt = dt; a.mode = mode; a.hidden = hidden; a.cu_seqlens = cu_seqlens; a.n_visual = n_visual; a.cu_vis = cu_vis;
   a.kept_idx = kept_idx; a.cu_kept = cu_kept; a.B = B; a.D = D; a.total_tokens = total_tokens; a.total_out = total_out;
@@ -263,7 +263,31 @@ int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* hidd
       if (st != D3TOM_OK) return st;
     }
   }
-  return launch_merge_finish(ctx, a, s);
+  st = launch_merge_finish(ctx, a, s);
+  if (st != D3TOM_OK || second == nullptr) return st;
+  a.hidden = second; a.hidden_out = second_out;       // same routing, second payload
+  return launch_merge_aggregate(ctx, a, s);
+}
+
+int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* hidden, const int32_t* cu_seqlens,
+                const int32_t* n_visual, const int32_t* cu_vis, const int32_t* kept_idx, const int32_t* cu_kept,
+                int B, int D, int total_tokens, int total_out, int max_visual, int max_kept, void* hidden_out,
+                const int32_t* cu_seqlens_out, int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
+                float* sim_debug, d3tom_stream stream) {
+  return merge_common(ctx, dt, mode, hidden, nullptr, cu_seqlens, n_visual, cu_vis, kept_idx, cu_kept, B, D,
+                      total_tokens, total_out, max_visual, max_kept, hidden_out, nullptr, cu_seqlens_out, assign,
+                      member_count, src_of_dst, sim_debug, static_cast<cudaStream_t>(stream));
+}
+
+int d3tom_merge_kv(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* k_cache, const void* v_cache,
+                   const int32_t* cu_seqlens, const int32_t* n_visual, const int32_t* cu_vis, const int32_t* kept_idx,
+                   const int32_t* cu_kept, int B, int D, int total_tokens, int total_out, int max_visual, int max_kept,
+                   void* k_out, void* v_out, const int32_t* cu_seqlens_out, int32_t* assign, int32_t* member_count,
+                   int32_t* src_of_dst, float* sim_debug, d3tom_stream stream) {
+  if (v_cache == nullptr || v_out == nullptr) return D3TOM_ERR_INVALID_ARG;
+  return merge_common(ctx, dt, mode, k_cache, v_cache, cu_seqlens, n_visual, cu_vis, kept_idx, cu_kept, B, D,
+                      total_tokens, total_out, max_visual, max_kept, k_out, v_out, cu_seqlens_out, assign,
+                      member_count, src_of_dst, sim_debug, static_cast<cudaStream_t>(stream));
 }
 
 int d3tom_proj_qkv(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_qkv, int total, int D, void* q,

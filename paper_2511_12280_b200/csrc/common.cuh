@@ -147,6 +147,7 @@ int launch_merge_prepare(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);   
 int launch_sim_simt(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);          // similarity + argmax, CUDA cores
 int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);            // similarity + argmax, tcgen05
 int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);      // members, aggregate, compact
+int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);   // aggregate, compact (lists already built)
 
 int launch_proj_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w, int total, int D,
                      void* q, void* k, void* v, cudaStream_t s);

@@ -511,6 +511,12 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
                                                    ctx->member_off, ctx->member_cursor, ctx->member_list,
                                                    ctx->heavy_slots, ctx->n_heavy, ctr_ints, bitmap_warps);
   D3TOM_LAUNCH_CHECK(ctx);
+  return launch_merge_aggregate(ctx, a, s);
+}
+
+// aggregation + compaction of a.hidden into a.hidden_out with the member lists the context holds
+// (may run again on another tensor of the same rows: the V cache after the K cache)
+int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   const int mean = a.mode == D3TOM_AGG_MEAN ? 1 : 0;
   if (a.total_out <= 0) return D3TOM_OK;
   const int vec = a.dt == D3TOM_FP32 ? 4 : 8;

@@ -366,3 +366,50 @@ def test_flop_model_is_sensitive_to_the_readings_it_pins():
     assert abs(fm.flops_d3tom(0.75, 4) / 1e12 - 109.12) > 0.5
     other = sum(fm.flops_step(orc.schedule_alpha(s, 32, 0.625, 0.875), 3, N, fm.N_VIS) for s in range(32)) / 32
     assert abs((fm.L_LAYERS * fm.flops_layer(N) + 31 * other) / 1e12 - 109.27) > 0.05
+
+
+# ------------------------------------------------------------------ KV-cache merge (Sec. 4.4)
+def test_merge_kv_equals_pure_python_brute_force():
+    r = rng(31)
+    V, P, D = 9, 3, 4
+    K = r.standard_normal((V + P, D)); Vv = r.standard_normal((V + P, D))
+    kept = np.array([1, 4, 7])
+    res = orc.merge_kv(K, Vv, [0, V + P], [V], [kept], orc.SUM, "fp32")
+    # brute force: cosine on K only, sums of K and V, dropped positions
+    k_new = {int(k): list(K[k]) for k in kept}; v_new = {int(k): list(Vv[k]) for k in kept}
+    for m in range(V):
+        if m in kept:
+            continue
+        best, arg = -2.0, None
+        for k in kept:
+            dot = sum(K[m][c] * K[k][c] for c in range(D))
+            cos = dot / math.sqrt(sum(x * x for x in K[m])) / math.sqrt(sum(x * x for x in K[k]))
+            if cos > best:
+                best, arg = cos, int(k)
+        for c in range(D):
+            k_new[arg][c] += K[m][c]; v_new[arg][c] += Vv[m][c]
+    want_k = np.array([k_new[int(k)] for k in kept] + [list(x) for x in K[V:]])
+    want_v = np.array([v_new[int(k)] for k in kept] + [list(x) for x in Vv[V:]])
+    assert np.allclose(res["k_out"], want_k.astype(np.float32), rtol=1e-6, atol=1e-6)
+    assert np.allclose(res["v_out"], want_v.astype(np.float32), rtol=1e-6, atol=1e-6)
+    assert res["k_out"].shape[0] == P + len(kept) and list(res["src_of_dst"]) == [1, 4, 7, 9, 10, 11]
+
+
+def test_merge_kv_routing_depends_on_keys_only_and_conserves_mass():
+    r = rng(32)
+    V, P, D = 40, 5, 8
+    K, Va, Vb = (r.standard_normal((V + P, D)).astype(np.float32).astype(np.float64) for _ in range(3))   # storage precision
+    kept = np.sort(r.choice(V, 7, replace=False))
+    a = orc.merge_kv(K, Va, [0, V + P], [V], [kept], orc.SUM, "fp32")
+    b = orc.merge_kv(K, Vb, [0, V + P], [V], [kept], orc.SUM, "fp32")
+    assert np.array_equal(a["assign"], b["assign"])                      # values never influence the routing
+    assert np.array_equal(a["assign"], orc.assign(K[:V], kept))          # it is the merge routing applied to K
+    # SUM conserves the column sums of both caches over the visual rows
+    assert np.allclose(a["k_out"][:7].sum(0), K[:V].sum(0), atol=1e-5)
+    assert np.allclose(a["v_out"][:7].sum(0), Va[:V].sum(0), atol=1e-5)
+    # MEAN divides both by 1 + members
+    m = orc.merge_kv(K, Va, [0, V + P], [V], [kept], orc.MEAN, "fp32")
+    assert np.allclose(m["v_out"][:7] * (1 + m["member_count"])[:, None], a["v_out"][:7], atol=1e-5)
+    # keeping everything is the identity on both caches
+    ident = orc.merge_kv(K, Va, [0, V + P], [V], [np.arange(V)], orc.SUM, "fp32")
+    assert np.array_equal(ident["k_out"], K) and np.array_equal(ident["v_out"], Va)
