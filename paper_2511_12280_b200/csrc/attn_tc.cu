@@ -110,7 +110,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       ptx::mbar_init(&p_lo[i], 4); ptx::mbar_init(&p_hi[i], 4);      // one arrival per softmax warp
       ptx::mbar_init(&o_final[i], 1);
     }
-    for (int s = 0; s < kKvSlots; ++s) { ptx::mbar_init(&kv_full[s], 1); ptx::mbar_init(&kv_empty[s], 1); }
+    for (int s = 0; s < kKvSlots; ++s) { ptx::mbar_init(&kv_full[s], 1); ptx::mbar_init(&kv_empty[s], 4 * n_qt); }   // freed by the softmax warps
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -184,7 +184,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (ok) {
           ptx::tc_fence_after_sync();
           for (int i = 0; i < n_qt; ++i) { issue_qk(i, 0); ptx::mma_commit(&s_full[i]); }
-          ptx::mma_commit(&kv_empty[0]);          // stage 0 held K_0 only: the producer may go on to stage 2
         }
         // Key tile j needs stage j+1 (V_j and K_(j+1)).  The softmax warps wait for that stage
         // before they announce P_j, so this thread has no load barrier of its own to check: every
@@ -208,7 +207,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
               ptx::mma_commit(&o_final[i]);
             }
           }
-          if (ok) ptx::mma_commit(&kv_empty[st]);   // frees stage j+1 once everything issued so far is done
         }
       }
     }
@@ -246,6 +244,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[i], j & 1, abort_flag, a.dev_status));
         if (!ok) break;
         ptx::tc_fence_after_sync();
+        // S_j of this tile is complete, so its QK^T has read K_j and, issued before it, the PV of the
+        // previous key tile has read V_(j-1): stage j is free once every softmax warp has seen that
+        // (a commit by the MMA thread would cost the tensor pipe an issue gap)
+        if (lane == 0) ptx::mbar_arrive(&kv_empty[j & 1]);
         // ---- the whole score row of this tile: 128 fp32 values, one TMEM lane
         uint32_t sr[kTile];
         ptx::tmem_ld32(t_s, sr);
