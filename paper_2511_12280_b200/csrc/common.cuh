@@ -28,6 +28,7 @@ struct d3tom_ctx {
   int32_t* member_list;         // [max_total_tokens] pruned positions grouped by destination slot
   int32_t* heavy_slots;         // [max_total_tokens / 32 + 1] kept tokens with 32 members or more
   int* n_heavy;                 // how many of them
+  int4* row_desc;               // [max_total_tokens] per output row: {source row, members or -1, list offset, request start}
   float* gemm_split_ws;         // [2 * sm_count][256][128] fp32 partial similarity tiles (K slices of a tile)
   int* gemm_split_counters;     // [2 * sm_count] slices done per tile; zero between launches
   int* dev_status;              // device status word

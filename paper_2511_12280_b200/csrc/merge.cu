@@ -174,12 +174,17 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
                const unsigned long long* __restrict__ best, int32_t* __restrict__ assign,
                int32_t* __restrict__ member_count, int32_t* __restrict__ member_off,
                int32_t* __restrict__ cursor, int32_t* __restrict__ member_list,
-               int32_t* __restrict__ heavy_slots, int* __restrict__ n_heavy, int ctr_ints, int bitmap_warps) {
+               int32_t* __restrict__ heavy_slots, int* __restrict__ n_heavy, int ctr_ints, int bitmap_warps,
+               const int32_t* __restrict__ cu_seqlens, const int32_t* __restrict__ cu_seqlens_out,
+               const int32_t* __restrict__ kept_idx, int4* __restrict__ row_desc) {
   extern __shared__ int dyn_s[];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int v0 = cu_vis[b], V = cu_vis[b + 1] - v0;
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
   const int pruned_base = v0 - k0;                 // pruned tokens of earlier requests
+  const int lo = cu_seqlens[b], out0 = cu_seqlens_out[b], n_out = cu_seqlens_out[b + 1] - out0;
+  // prompt / response rows are copied: member count -1 marks them
+  for (int r = kb + tid; r < n_out; r += kMemberThreads) row_desc[out0 + r] = make_int4(lo + V + (r - kb), -1, 0, lo);
   int* ctr = kb <= ctr_ints ? dyn_s : cursor + k0;
   unsigned* bitmaps = reinterpret_cast<unsigned*>(dyn_s + ctr_ints);
   __shared__ int warp_tot[32];
@@ -227,6 +232,8 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
       member_off[k0 + s] = pruned_base + excl;
       ctr[s] = pruned_base + excl;
       if (c >= kHeavy) heavy_slots[atomicAdd(n_heavy, 1)] = k0 + s;
+      // what the aggregation needs to know about this output row, in one 16-byte record
+      row_desc[out0 + s] = make_int4(lo + kept_idx[k0 + s], c, pruned_base + excl, lo);
     }
     __syncthreads();
     if (tid == 0) carry += chunk_total;
@@ -329,7 +336,8 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
                          int chunks, int total_out, int heavy_blocks, int mean,
                          const int32_t* __restrict__ member_count, const int32_t* __restrict__ member_off,
                          const int32_t* __restrict__ member_list, const int32_t* __restrict__ heavy_slots,
-                         const int* __restrict__ n_heavy, T* __restrict__ hidden_out, int32_t* __restrict__ src_of_dst) {
+                         const int* __restrict__ n_heavy, const int4* __restrict__ row_desc, T* __restrict__ hidden_out,
+                         int32_t* __restrict__ src_of_dst) {
   constexpr int kVec = Storage<T>::kVec;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float acc[kVec];
@@ -383,10 +391,9 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
   const int gw = ((int)blockIdx.x - heavy_blocks) * kAggWarps + warp;
   const int row = gw / groups, cg = gw - row * groups;
   if (row >= total_out) return;                                 // whole warp
-  const int b = find_segment(cu_seqlens_out, B, row);
-  const int r = row - cu_seqlens_out[b];
-  const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
-  const int lo = cu_seqlens[b], Vb = n_visual[b];
+  const int4 desc = row_desc[row];                             // {source row, members (-1: copy), list offset, request's first row}
+  const int cnt = desc.y, off = desc.z, lo = desc.w;
+  const int pos = desc.x - lo;                                  // position in the request
   int col[kAggCpw];
   bool live[kAggCpw];
 #pragma unroll
@@ -397,21 +404,16 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
   }
   const T* req = hidden + (size_t)lo * D;
   T* dst = hidden_out + (size_t)row * D;
+  if (cg == 0 && lane == 0) src_of_dst[row] = desc.x;
 
-  if (r >= kb) {                                                // prompt / response row: copy
-    const int src_row = Vb + (r - kb);
+  if (cnt < 0) {                                                // prompt / response row: copy
     uint4 raw[kAggCpw];
 #pragma unroll
-    for (int j = 0; j < kAggCpw; ++j) raw[j] = *reinterpret_cast<const uint4*>(req + (size_t)src_row * D + col[j]);
+    for (int j = 0; j < kAggCpw; ++j) raw[j] = *reinterpret_cast<const uint4*>(req + (size_t)pos * D + col[j]);
 #pragma unroll
     for (int j = 0; j < kAggCpw; ++j) if (live[j]) *reinterpret_cast<uint4*>(dst + col[j]) = raw[j];
-    if (cg == 0 && lane == 0) src_of_dst[row] = lo + src_row;
     return;
   }
-
-  const int pos = kept_idx[k0 + r];
-  const int cnt = member_count[k0 + r];
-  const int off = member_off[k0 + r];
   if (cnt >= kHeavy) return;                                    // a heavy block does this row
   // lane t ends up holding the t-th row to add: the kept row, then the members by ascending
   // position (distinct values, ranked by counting the smaller ones)
@@ -454,7 +456,6 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
       for (int e = 0; e < kVec; ++e) accs[j][e] *= inv_denom;
       Storage<T>::store(dst + col[j], accs[j]);
     }
-  if (cg == 0 && lane == 0) src_of_dst[row] = lo + pos;
 }
 
 }  // namespace
@@ -509,7 +510,8 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   D3TOM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->n_heavy, 0, sizeof(int), s));
   members_kernel<<<a.B, kMemberThreads, smem, s>>>(a.cu_vis, a.cu_kept, ctx->best, a.assign, a.member_count,
                                                    ctx->member_off, ctx->member_cursor, ctx->member_list,
-                                                   ctx->heavy_slots, ctx->n_heavy, ctr_ints, bitmap_warps);
+                                                   ctx->heavy_slots, ctx->n_heavy, ctr_ints, bitmap_warps, a.cu_seqlens, a.cu_seqlens_out,
+                                                   a.kept_idx, ctx->row_desc);
   D3TOM_LAUNCH_CHECK(ctx);
   return launch_merge_aggregate(ctx, a, s);
 }
@@ -532,12 +534,12 @@ int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
     aggregate_compact_kernel<float><<<blocks, kAggWarps * 32, 0, s>>>(
         static_cast<const float*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out, a.B, a.D,
         chunks, a.total_out, heavy_blocks, mean, a.member_count, ctx->member_off, ctx->member_list, ctx->heavy_slots,
-        ctx->n_heavy, static_cast<float*>(a.hidden_out), a.src_of_dst);
+        ctx->n_heavy, ctx->row_desc, static_cast<float*>(a.hidden_out), a.src_of_dst);
   else
     aggregate_compact_kernel<__nv_bfloat16><<<blocks, kAggWarps * 32, 0, s>>>(
         static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out,
         a.B, a.D, chunks, a.total_out, heavy_blocks, mean, a.member_count, ctx->member_off, ctx->member_list,
-        ctx->heavy_slots, ctx->n_heavy, static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
+        ctx->heavy_slots, ctx->n_heavy, ctx->row_desc, static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }
