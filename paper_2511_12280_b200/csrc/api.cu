@@ -29,7 +29,7 @@ void free_all(d3tom_ctx* c) {
   cudaFree(c->score_scratch); cudaFree(c->lse_scratch); cudaFree(c->imp_partial); cudaFree(c->imp_counters);
   cudaFree(c->inv_norm);
   cudaFree(c->inv_norm_kept); cudaFree(c->kept_rows); cudaFree(c->best); cudaFree(c->member_off);
-  cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->heavy_slots); cudaFree(c->n_heavy); cudaFree(c->row_desc);
+  cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->heavy_slots); cudaFree(c->n_heavy); cudaFree(c->row_desc); cudaFree(c->agg_counter);
   cudaFree(c->gemm_split_ws); cudaFree(c->gemm_split_counters); cudaFree(c->dev_status);
 }
 
@@ -84,6 +84,7 @@ int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (st == D3TOM_OK) st = alloc(c, &c->heavy_slots, T / 32 + 1);
   if (st == D3TOM_OK) st = alloc(c, &c->n_heavy, 1);
   if (st == D3TOM_OK) st = alloc(c, &c->row_desc, T);
+  if (st == D3TOM_OK) st = alloc(c, &c->agg_counter, 1);
   if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_ws, (size_t)2 * c->sm_count * 128 * 256);
   if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_counters, (size_t)2 * c->sm_count);
   if (st == D3TOM_OK && cudaMemset(c->gemm_split_counters, 0, 2 * c->sm_count * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;

@@ -28,6 +28,7 @@ struct d3tom_ctx {
   int32_t* member_list;         // [max_total_tokens] pruned positions grouped by destination slot
   int32_t* heavy_slots;         // [max_total_tokens / 32 + 1] kept tokens with 32 members or more
   int* n_heavy;                 // how many of them
+  int* agg_counter;             // work counter of the streaming aggregation; zeroed before each launch
   int4* row_desc;               // [max_total_tokens] per output row: {source row, members or -1, list offset, request start}
   float* gemm_split_ws;         // [2 * sm_count][256][128] fp32 partial similarity tiles (K slices of a tile)
   int* gemm_split_counters;     // [2 * sm_count] slices done per tile; zero between launches
@@ -149,6 +150,7 @@ int launch_sim_simt(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);        
 int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);            // similarity + argmax, tcgen05
 int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);      // members, aggregate, compact
 int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);   // aggregate, compact (lists already built)
+int launch_merge_aggregate_stream(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);   // the same as a bulk-copy pipeline
 
 int launch_proj_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w, int total, int D,
                      void* q, void* k, void* v, cudaStream_t s);

@@ -521,6 +521,10 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
 int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   const int mean = a.mode == D3TOM_AGG_MEAN ? 1 : 0;
   if (a.total_out <= 0) return D3TOM_OK;
+  {   // the streaming pipeline takes every row size it supports; the kernel below is the general one
+    const int st = launch_merge_aggregate_stream(ctx, a, s);
+    if (st != D3TOM_ERR_UNSUPPORTED) return st;
+  }
   const int vec = a.dt == D3TOM_FP32 ? 4 : 8;
   const int chunks = ceil_div(a.D, 32 * vec);                       // 512-byte chunks per row
   const long long warps = (long long)a.total_out * ceil_div(chunks, kAggCpw);

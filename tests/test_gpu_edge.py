@@ -40,6 +40,15 @@ def test_lengths_around_tile_boundaries():
     pu.check_step(small(reqs=reqs, post=1))
 
 
+def test_many_rows_fp32_take_the_streaming_aggregation():
+    # more than 4096 output rows: the aggregation runs as the bulk-copy pipeline (bf16 is covered by the ragged
+    # serving config); narrow rows keep the oracle cheap
+    reqs = [dict(V=3000, P=40, O=12, n_dec=3, r=0.8), dict(V=2600, P=9, O=8, n_dec=2, r=0.7)]
+    w = wl.make_workload("rows", "fp32", 2, 32, 13, 16, reqs, post_layers=0)
+    pu.check_step(w, full_attention=False, n_sample_rows=8)
+    pu.check_step(w, mode=B_.AGG_SUM, full_attention=False, n_sample_rows=8)
+
+
 def test_keep_ratio_one_is_identity():
     w = small(post=0)
     step = pu.make_step(w, keep_count=list(w.n_visual), sim_debug=False)
