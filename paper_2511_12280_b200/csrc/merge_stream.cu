@@ -19,7 +19,7 @@ namespace {
 constexpr int kConsumerWarps = 4;
 constexpr int kStreamThreads = 32 * (1 + kConsumerWarps);
 constexpr int kMaxSlots = 32;
-constexpr int kRingBytes = 64 * 1024;
+constexpr int kRingBytes = 32 * 1024;
 constexpr int kMaxVecPerThread = 4;        // 16-byte vectors of a segment per consumer thread
 constexpr int kStreamMinRows = 4096;       // fewer output rows than this go to the plain kernel
 constexpr int kHeavyList = 32;             // lists of this many members or more are already sorted in memory
@@ -205,7 +205,8 @@ int launch_merge_aggregate_stream(d3tom_ctx* ctx, const MergeArgs& a, cudaStream
   D3TOM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->agg_counter, 0, sizeof(int), s));
   const size_t smem = (size_t)slots * seg + 128;
   const long long items = (long long)a.total_out * splits;
-  long long grid = 3LL * ctx->sm_count;                 // three CTAs fit one SM (64 KB of ring each)
+  long long grid = 6LL * ctx->sm_count;                 // six CTAs fit one SM (32 KB of ring each): what limits the
+                                                        // pipeline is the rate at which one producer lane issues copies
   if (grid > items) grid = items;
   if (a.dt == D3TOM_FP32) {
     D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(aggregate_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes + 128));
