@@ -54,9 +54,26 @@ template <int BN> struct GemmSmem {
 template <int BN, int EPI>
 struct TileCoord {
   int m0, n0, a_row, b_row, b, Vb, kb, v0, k0;
+  const int* prefix;      // similarity with a ragged batch: tiles before request b (shared memory), or null
   __device__ __forceinline__ bool set(const GemmParams& p, int t) {
-    const int mi = t % p.m_tiles, rest = t / p.m_tiles;
-    const int ni = rest % p.n_tiles;
+    int mi, ni;
+    if (EPI == kEpiSim && prefix != nullptr) {
+      // only the tiles that exist are numbered: request b owns [prefix[b], prefix[b + 1]), M fastest
+      b = 0;
+      while (prefix[b + 1] <= t) ++b;
+      const int local = t - prefix[b];
+      v0 = p.cu_vis[b]; Vb = p.cu_vis[b + 1] - v0;
+      k0 = p.cu_kept[b]; kb = p.cu_kept[b + 1] - k0;
+      const int mt = (Vb + kBM - 1) / kBM;
+      mi = local % mt; ni = local / mt;
+      m0 = mi * kBM; n0 = ni * BN;
+      a_row = p.cu_seqlens[b] + m0;
+      b_row = k0 + n0;
+      return true;
+    }
+    mi = t % p.m_tiles;
+    const int rest = t / p.m_tiles;
+    ni = rest % p.n_tiles;
     b = rest / p.n_tiles;
     m0 = mi * kBM; n0 = ni * BN; a_row = m0; b_row = n0;
     Vb = kb = v0 = k0 = 0;
@@ -70,6 +87,8 @@ struct TileCoord {
     return true;
   }
 };
+
+constexpr int kMaxPrefixBatch = 64;     // ragged batches up to this many requests number only the tiles that exist
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -89,7 +108,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   float* ink_s = reinterpret_cast<float*>(smem + kStages * (S::kABytes + S::kBBytes) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_units = p.m_tiles * p.n_tiles * p.batch * p.k_splits;   // a unit = one tile, or one K slice of a tile
+  int total_units = p.m_tiles * p.n_tiles * p.batch * p.k_splits;   // a unit = one tile, or one K slice of a tile
+  // A batch of requests of different sizes: the bounding grid (batch x largest request) is mostly holes, and
+  // walking it leaves the SMs unevenly loaded.  Every CTA numbers the tiles that exist (a prefix over requests).
+  __shared__ int tile_prefix[kMaxPrefixBatch + 1];
+  const bool use_prefix = EPI == kEpiSim && p.batch > 1 && p.batch <= kMaxPrefixBatch;
+  if (use_prefix) {
+    if (threadIdx.x == 0) {
+      int run = 0;
+      for (int b = 0; b < p.batch; ++b) {
+        tile_prefix[b] = run;
+        const int Vb = p.cu_vis[b + 1] - p.cu_vis[b], kb = p.cu_kept[b + 1] - p.cu_kept[b];
+        if (kb < Vb) run += ((Vb + kBM - 1) / kBM) * ((kb + BN - 1) / BN);
+      }
+      tile_prefix[p.batch] = run;
+    }
+    __syncthreads();
+    total_units = tile_prefix[p.batch] * p.k_splits;
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }   // A and B loaders
@@ -103,6 +139,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   TileCoord<BN, EPI> tc;
+  tc.prefix = use_prefix ? tile_prefix : nullptr;
 
   if (warp == 0 || warp == 6) {
     // ------------------------------------------------------------ TMA producers: warp 0 streams A, warp 6 streams B
