@@ -49,6 +49,14 @@ def test_many_rows_fp32_take_the_streaming_aggregation():
     pu.check_step(w, mode=B_.AGG_SUM, full_attention=False, n_sample_rows=8)
 
 
+def test_single_request_single_tile_ctas_with_deciders():
+    # one request, few heads: every 128-row tile becomes a CTA of its own (the decider rows included)
+    w = small(H=4, reqs=[dict(V=520, P=40, O=40, n_dec=7, r=0.25)], post=1)
+    pu.check_step(w)
+    w = small(H=2, dh=64, reqs=[dict(V=900, P=11, O=30, n_dec=30, r=0.5)], post=1)
+    pu.check_step(w, mode=B_.AGG_SUM)
+
+
 def test_keep_ratio_one_is_identity():
     w = small(post=0)
     step = pu.make_step(w, keep_count=list(w.n_visual), sim_debug=False)
