@@ -222,6 +222,7 @@ def main():
     ap.add_argument("--config", default="C2", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
     ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "step"],
                     help="profiling aid: after one full step, run just this call --steps times and exit")
     args = ap.parse_args()
@@ -324,12 +325,24 @@ def main():
         return replicas.max_over_ranks(x, dev)
 
     counter = {"i": 0, "launches": 0}
+    # one CUDA graph per problem: a step is then one graph launch (the kernels and their order are unchanged)
+    graphs = None
+    if not args.no_graph and args.only is None:
+        graphs = []
+        for i in range(n_prob):
+            step.use_problem(probs[i])
+            graphs.append(step.capture(qs[i], k, v, w_post))
+        step.use_problem(probs[n_prob // 2])
+    config["launch"] = "cuda graph replay, one per step" if graphs is not None else "host launches"
 
     def run():
         i = counter["i"] % n_prob
         counter["i"] += 1
         step.use_problem(probs[i])
         counter["launches"] += step.launches_per_step()
+        if graphs is not None:
+            graphs[i].replay()
+            return step.layer_out[-1] if step.n_post else step.hidden_out
         return step.run(qs[i], k, v, w_post)
 
     if args.only is not None:
@@ -398,13 +411,23 @@ def main():
 
     # ---- end to end through the C ABI with host buffers: H2D of Q,K,V, the step, D2H of the result
     e2e_bytes = {"h2d": 0, "d2h": 0, "n": 0}
+    e2e_graphs = None
+    if graphs is not None:          # the same step recorded on the buffer that the host copy fills
+        e2e_graphs = []
+        for i in range(n_prob):
+            step.use_problem(probs[i])
+            e2e_graphs.append(step.capture(q_stage, k, v, w_post))
 
     def e2e():
         i = counter["i"] % n_prob
         counter["i"] += 1
         step.use_problem(probs[i])
         q_stage.copy_(q_hs[i], non_blocking=True); k.copy_(k_h, non_blocking=True); v.copy_(v_h, non_blocking=True)
-        y = step.run(q_stage, k, v, w_post)
+        if e2e_graphs is not None:
+            e2e_graphs[i].replay()
+            y = step.layer_out[-1] if step.n_post else step.hidden_out
+        else:
+            y = step.run(q_stage, k, v, w_post)
         out_h[:step.total_out].copy_(y[:step.total_out], non_blocking=True)
         e2e_bytes["h2d"] += 3 * q_stage.numel() * q_stage.element_size()
         e2e_bytes["d2h"] += step.total_out * step.D * q_stage.element_size()

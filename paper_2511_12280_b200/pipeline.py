@@ -126,6 +126,21 @@ class MergeLayerStep:
             x = self.layer_out[l]
         return x
 
+    def capture(self, q, k, v, w_post: Optional[Sequence[torch.Tensor]] = None):
+        """Records run(q, k, v, w_post) for the current problem into a CUDA graph and returns it
+        (call .replay() to enqueue the whole step with one launch).  The graph reads and writes
+        the same buffers as run(); q, k, v may be refilled between replays.  One untimed run is
+        made first on a side stream, as capture requires."""
+        side = torch.cuda.Stream(device=self.dev)
+        side.wait_stream(torch.cuda.current_stream(self.dev))
+        with torch.cuda.stream(side):
+            self.run(q, k, v, w_post)
+        torch.cuda.current_stream(self.dev).wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(q, k, v, w_post)
+        return graph
+
     def launches_per_step(self) -> int:
         """Kernels of this library launched by one run(): attention 1 + importance finish 1,
         select 1, merge 1 (prepare) + 1 (similarity, when something is pruned) + 2 (members,
