@@ -57,6 +57,13 @@ def test_single_request_single_tile_ctas_with_deciders():
     pu.check_step(w, mode=B_.AGG_SUM)
 
 
+def test_kept_set_larger_than_the_shared_memory_counters():
+    # more than 12288 kept tokens in one request: the member counters live in global memory, the bitmap of a
+    # sorting warp spans 13000 positions, and select stages 13000 keys
+    w = small(H=1, dh=64, reqs=[dict(V=13000, P=8, O=8, n_dec=3, r=0.97)], post=0)
+    pu.check_step(w, full_attention=False, n_sample_rows=6)
+
+
 def test_keep_ratio_one_is_identity():
     w = small(post=0)
     step = pu.make_step(w, keep_count=list(w.n_visual), sim_debug=False)
