@@ -84,7 +84,8 @@ int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (st == D3TOM_OK) st = alloc(c, &c->heavy_slots, T / 32 + 1);
   if (st == D3TOM_OK) st = alloc(c, &c->n_heavy, 1);
   if (st == D3TOM_OK) st = alloc(c, &c->row_desc, T);
-  if (st == D3TOM_OK) st = alloc(c, &c->agg_counter, 1);
+  if (st == D3TOM_OK) st = alloc(c, &c->agg_counter, 2);
+  if (st == D3TOM_OK && cudaMemset(c->agg_counter, 0, 2 * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_ws, (size_t)2 * c->sm_count * 128 * 256);
   if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_counters, (size_t)2 * c->sm_count);
   if (st == D3TOM_OK && cudaMemset(c->gemm_split_counters, 0, 2 * c->sm_count * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;

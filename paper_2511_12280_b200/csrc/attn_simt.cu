@@ -18,6 +18,7 @@ constexpr int kRowsPerBlock = 8;   // warps per block
 template <typename T>
 __global__ void __launch_bounds__(kRowsPerBlock * 32)
 attn_simt_kernel(AttnArgs a) {
+  grid_dependency_enter();
   const int b = blockIdx.z, h = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int lo = a.cu_seqlens[b], n = a.cu_seqlens[b + 1] - lo;
@@ -102,6 +103,7 @@ importance_finish_kernel(const float* __restrict__ score, const float2* __restri
                          const int32_t* __restrict__ cu_vis, int max_deciders, int vis_stride, float scale_log2,
                          float* __restrict__ partial, int partial_stride, int H, int* __restrict__ counters,
                          float* __restrict__ importance) {
+  grid_dependency_enter();
   const int b = blockIdx.z, h = blockIdx.y;
   const int Vb = n_visual[b];
   if ((int)blockIdx.x * kImpThreads >= Vb) return;              // uniform: no key of this request in the range
@@ -148,9 +150,8 @@ importance_finish_kernel(const float* __restrict__ score, const float2* __restri
 
 int launch_attn_simt(d3tom_ctx* ctx, d3tom_dtype dt, const AttnArgs& a, cudaStream_t s) {
   dim3 grid(ceil_div(a.max_seqlen, kRowsPerBlock), a.H, a.B);
-  if (dt == D3TOM_FP32) attn_simt_kernel<float><<<grid, kRowsPerBlock * 32, 0, s>>>(a);
-  else attn_simt_kernel<__nv_bfloat16><<<grid, kRowsPerBlock * 32, 0, s>>>(a);
-  D3TOM_LAUNCH_CHECK(ctx);
+  if (dt == D3TOM_FP32) D3TOM_CUDA_TRY(ctx, launch_serialized(attn_simt_kernel<float>, grid, kRowsPerBlock * 32, 0, s, a));
+  else D3TOM_CUDA_TRY(ctx, launch_serialized(attn_simt_kernel<__nv_bfloat16>, grid, kRowsPerBlock * 32, 0, s, a));
   return D3TOM_OK;
 }
 
@@ -158,9 +159,8 @@ int launch_importance_finish(d3tom_ctx* ctx, const AttnArgs& a, int max_visual, 
                              const int32_t* cu_vis, cudaStream_t s) {
   if (max_visual <= 0) return D3TOM_OK;
   dim3 grid(ceil_div(max_visual, kImpThreads), a.H, a.B);
-  importance_finish_kernel<<<grid, kImpThreads, 0, s>>>(a.score_scratch, a.lse_scratch, a.n_visual, a.cu_deciders, cu_vis,
-                                                        a.max_deciders, a.vis_stride, a.scale_log2, ctx->imp_partial,
-                                                        ctx->lim.max_total_tokens, a.H, ctx->imp_counters, importance);
-  D3TOM_LAUNCH_CHECK(ctx);
+  D3TOM_CUDA_TRY(ctx, launch_serialized(importance_finish_kernel, grid, kImpThreads, 0, s, a.score_scratch, a.lse_scratch,
+                                        a.n_visual, a.cu_deciders, cu_vis, a.max_deciders, a.vis_stride, a.scale_log2,
+                                        ctx->imp_partial, ctx->lim.max_total_tokens, a.H, ctx->imp_counters, importance));
   return D3TOM_OK;
 }

@@ -74,6 +74,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   // (one head's K/V stay hot in L2), query blocks from the end.  Items from `split_from` on are cut
   // into two CTAs of one 128-row tile each: the host does that to the items of an incomplete last
   // wave, which then costs the time of a single tile instead of a pair.
+  grid_dependency_enter();
   const int items = a.H * a.nqb, per_req = items + (items - a.split_from);
   const int b = (int)blockIdx.x / per_req, lin = (int)blockIdx.x - b * per_req;
   int item = lin, half = -1;
@@ -400,7 +401,7 @@ int launch(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
     else if (items > sms && rest > 0 && 2 * rest <= sms) k.split_from = items - rest;   // incomplete last wave
   }
   const int grid = a.B * (items + (items - k.split_from));
-  attn_tc_kernel<DH><<<grid, kAttnThreads, AttnSmem<DH>::kBytes, s>>>(tq, tk, tv, k);
+  D3TOM_CUDA_TRY(ctx, launch_serialized(attn_tc_kernel<DH>, grid, kAttnThreads, AttnSmem<DH>::kBytes, s, tq, tk, tv, k));
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }

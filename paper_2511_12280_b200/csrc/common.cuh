@@ -28,7 +28,7 @@ struct d3tom_ctx {
   int32_t* member_list;         // [max_total_tokens] pruned positions grouped by destination slot
   int32_t* heavy_slots;         // [max_total_tokens / 32 + 1] kept tokens with 32 members or more
   int* n_heavy;                 // how many of them
-  int* agg_counter;             // work counter of the streaming aggregation; zeroed before each launch
+  int* agg_counter;             // [2] work and exit counters of the streaming aggregation; the kernel leaves them at zero
   int4* row_desc;               // [max_total_tokens] per output row: {source row, members or -1, list offset, request start}
   float* gemm_split_ws;         // [2 * sm_count][256][128] fp32 partial similarity tiles (K slices of a tile)
   int* gemm_split_counters;     // [2 * sm_count] slices done per tile; zero between launches
@@ -51,6 +51,31 @@ static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // ------------------------------------------------------------------ device helpers
 #ifdef __CUDACC__
+
+// Every kernel of the library is launched with programmatic stream serialization: its CTAs may become resident while
+// the kernel before it in the stream is still draining, which hides the launch latency between the many short
+// kernels of a step.  A kernel therefore opens with grid_dependency_enter(), BEFORE it touches global memory: it waits
+// until every earlier kernel has completed and its writes are visible, and only then lets the next kernel's CTAs be
+// scheduled (releasing before the wait let several kernels ahead pile up as waiting CTAs; measured no faster).
+// A kernel with on-chip set-up that needs no global memory does that set-up before the wait.
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_enter() {
+  grid_dependency_wait();
+  grid_dependency_release();
+}
+
+template <typename... Params, typename... Args>
+inline cudaError_t launch_serialized(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                     Args&&... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
 
 // largest b in [0, B) with cu[b] <= idx  (cu ascending, cu[0] = 0)
 __device__ __forceinline__ int find_segment(const int32_t* __restrict__ cu, int B, int idx) {

@@ -108,6 +108,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   float* ink_s = reinterpret_cast<float*>(smem + kStages * (S::kABytes + S::kBBytes) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // barriers and tensor memory first (on-chip only), then wait for the kernels before this one
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }   // A and B loaders
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }   // one arrival per epilogue warp
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 2) { ptx::tmem_alloc(tmem_slot, 2 * S::kAccStride); ptx::tmem_relinquish(); }
+  grid_dependency_wait();
+  grid_dependency_release();
   int total_units = p.m_tiles * p.n_tiles * p.batch * p.k_splits;   // a unit = one tile, or one K slice of a tile
   // A batch of requests of different sizes: the bounding grid (batch x largest request) is mostly holes, and
   // walking it leaves the SMs unevenly loaded.  Every CTA numbers the tiles that exist (a prefix over requests).
@@ -123,20 +133,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
       tile_prefix[p.batch] = run;
     }
-    __syncthreads();
-    total_units = tile_prefix[p.batch] * p.k_splits;
   }
 
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }   // A and B loaders
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 4); }   // one arrival per epilogue warp
-    *abort_flag = 0;
-    ptx::fence_mbar_init();
-  }
-  if (warp == 2) { ptx::tmem_alloc(tmem_slot, 2 * S::kAccStride); ptx::tmem_relinquish(); }
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
+  if (use_prefix) total_units = tile_prefix[p.batch] * p.k_splits;
   const uint32_t tmem_base = *tmem_slot;
   TileCoord<BN, EPI> tc;
   tc.prefix = use_prefix ? tile_prefix : nullptr;
@@ -368,8 +370,7 @@ int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, co
   const int grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);          // persistent: one CTA per SM
   D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            GemmSmem<BN>::kBytes));
-  gemm_tc_kernel<BN, EPI><<<grid, kGemmThreads, GemmSmem<BN>::kBytes, s>>>(ta, tb, p);
-  D3TOM_LAUNCH_CHECK(ctx);
+  D3TOM_CUDA_TRY(ctx, launch_serialized(gemm_tc_kernel<BN, EPI>, grid, kGemmThreads, GemmSmem<BN>::kBytes, s, ta, tb, p));
   return D3TOM_OK;
 }
 

@@ -46,8 +46,10 @@ prepare_rows_kernel(const T* __restrict__ hidden, const int32_t* __restrict__ cu
                     const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ kept_idx,
                     const int32_t* __restrict__ cu_kept, int D, int32_t* __restrict__ assign,
                     unsigned long long* __restrict__ best, float* __restrict__ inv_norm,
-                    float* __restrict__ inv_norm_kept, T* __restrict__ kept_rows) {
+                    float* __restrict__ inv_norm_kept, T* __restrict__ kept_rows, int* __restrict__ n_heavy) {
   constexpr int kVec = Storage<T>::kVec;
+  grid_dependency_enter();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *n_heavy = 0;   // counted by the members kernel, two launches on
   const int b = blockIdx.y, lane = threadIdx.x & 31;
   const int m = blockIdx.x * kPrepWarps + (threadIdx.x >> 5);
   const int v0 = cu_vis[b];
@@ -118,6 +120,7 @@ sim_simt_kernel(const T* __restrict__ hidden, const T* __restrict__ kept_rows,
                 const float* __restrict__ inv_norm, const float* __restrict__ inv_norm_kept,
                 int D, int max_kept, unsigned long long* __restrict__ best, float* __restrict__ sim_debug) {
   constexpr int kVec = Storage<T>::kVec;
+  grid_dependency_enter();
   const int b = blockIdx.y, m = blockIdx.x;
   const int v0 = cu_vis[b];
   if (m >= cu_vis[b + 1] - v0) return;
@@ -178,6 +181,7 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
                const int32_t* __restrict__ cu_seqlens, const int32_t* __restrict__ cu_seqlens_out,
                const int32_t* __restrict__ kept_idx, int4* __restrict__ row_desc) {
   extern __shared__ int dyn_s[];
+  grid_dependency_enter();
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int v0 = cu_vis[b], V = cu_vis[b + 1] - v0;
   const int k0 = cu_kept[b], kb = cu_kept[b + 1] - k0;
@@ -339,6 +343,7 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
                          const int* __restrict__ n_heavy, const int4* __restrict__ row_desc, T* __restrict__ hidden_out,
                          int32_t* __restrict__ src_of_dst) {
   constexpr int kVec = Storage<T>::kVec;
+  grid_dependency_enter();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float acc[kVec];
 #pragma unroll
@@ -463,33 +468,31 @@ aggregate_compact_kernel(const T* __restrict__ hidden, const int32_t* __restrict
 int launch_merge_prepare(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   dim3 grid(ceil_div(a.max_visual, kPrepWarps), a.B);
   if (a.dt == D3TOM_FP32)
-    prepare_rows_kernel<float><<<grid, kPrepWarps * 32, 0, s>>>(static_cast<const float*>(a.hidden), a.cu_seqlens, a.cu_vis,
-                                                               a.kept_idx, a.cu_kept, a.D, a.assign, ctx->best,
-                                                               ctx->inv_norm, ctx->inv_norm_kept,
-                                                               static_cast<float*>(ctx->kept_rows));
+    D3TOM_CUDA_TRY(ctx, launch_serialized(prepare_rows_kernel<float>, grid, kPrepWarps * 32, 0, s,
+                                          static_cast<const float*>(a.hidden), a.cu_seqlens, a.cu_vis, a.kept_idx,
+                                          a.cu_kept, a.D, a.assign, ctx->best, ctx->inv_norm, ctx->inv_norm_kept,
+                                          static_cast<float*>(ctx->kept_rows), ctx->n_heavy));
   else
-    prepare_rows_kernel<__nv_bfloat16><<<grid, kPrepWarps * 32, 0, s>>>(static_cast<const __nv_bfloat16*>(a.hidden),
-                                                                       a.cu_seqlens, a.cu_vis, a.kept_idx, a.cu_kept, a.D,
-                                                                       a.assign, ctx->best, ctx->inv_norm,
-                                                                       ctx->inv_norm_kept,
-                                                                       static_cast<__nv_bfloat16*>(ctx->kept_rows));
-  D3TOM_LAUNCH_CHECK(ctx);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(prepare_rows_kernel<__nv_bfloat16>, grid, kPrepWarps * 32, 0, s,
+                                          static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.cu_vis,
+                                          a.kept_idx, a.cu_kept, a.D, a.assign, ctx->best, ctx->inv_norm,
+                                          ctx->inv_norm_kept, static_cast<__nv_bfloat16*>(ctx->kept_rows), ctx->n_heavy));
   return D3TOM_OK;
 }
 
 int launch_sim_simt(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   dim3 grid(a.max_visual, a.B);
   if (a.dt == D3TOM_FP32)
-    sim_simt_kernel<float><<<grid, 256, 0, s>>>(static_cast<const float*>(a.hidden),
-                                                static_cast<const float*>(ctx->kept_rows), a.cu_seqlens, a.cu_vis,
-                                                a.cu_kept, a.assign, ctx->inv_norm, ctx->inv_norm_kept, a.D,
-                                                a.max_kept, ctx->best, a.sim_debug);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(sim_simt_kernel<float>, grid, 256, 0, s, static_cast<const float*>(a.hidden),
+                                          static_cast<const float*>(ctx->kept_rows), a.cu_seqlens, a.cu_vis, a.cu_kept,
+                                          a.assign, ctx->inv_norm, ctx->inv_norm_kept, a.D, a.max_kept, ctx->best,
+                                          a.sim_debug));
   else
-    sim_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(a.hidden),
-                                                        static_cast<const __nv_bfloat16*>(ctx->kept_rows),
-                                                        a.cu_seqlens, a.cu_vis, a.cu_kept, a.assign, ctx->inv_norm,
-                                                        ctx->inv_norm_kept, a.D, a.max_kept, ctx->best, a.sim_debug);
-  D3TOM_LAUNCH_CHECK(ctx);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(sim_simt_kernel<__nv_bfloat16>, grid, 256, 0, s,
+                                          static_cast<const __nv_bfloat16*>(a.hidden),
+                                          static_cast<const __nv_bfloat16*>(ctx->kept_rows), a.cu_seqlens, a.cu_vis,
+                                          a.cu_kept, a.assign, ctx->inv_norm, ctx->inv_norm_kept, a.D, a.max_kept,
+                                          ctx->best, a.sim_debug));
   return D3TOM_OK;
 }
 
@@ -507,12 +510,12 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   if (bitmap_warps > kMemberThreads / 32) bitmap_warps = kMemberThreads / 32;
   if (bitmap_warps < 1) return D3TOM_ERR_UNSUPPORTED;              // more than 512 Ki visual tokens in one request
   const size_t smem = (size_t)ctr_ints * sizeof(int) + (size_t)bitmap_warps * words * 4;
-  D3TOM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->n_heavy, 0, sizeof(int), s));
-  members_kernel<<<a.B, kMemberThreads, smem, s>>>(a.cu_vis, a.cu_kept, ctx->best, a.assign, a.member_count,
-                                                   ctx->member_off, ctx->member_cursor, ctx->member_list,
-                                                   ctx->heavy_slots, ctx->n_heavy, ctr_ints, bitmap_warps, a.cu_seqlens, a.cu_seqlens_out,
-                                                   a.kept_idx, ctx->row_desc);
-  D3TOM_LAUNCH_CHECK(ctx);
+  // the count of heavy kept tokens is zeroed by the prepare kernel, which runs whenever there are visual tokens
+  if (a.max_visual <= 0) D3TOM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->n_heavy, 0, sizeof(int), s));
+  D3TOM_CUDA_TRY(ctx, launch_serialized(members_kernel, a.B, kMemberThreads, smem, s, a.cu_vis, a.cu_kept, ctx->best, a.assign,
+                                        a.member_count, ctx->member_off, ctx->member_cursor, ctx->member_list,
+                                        ctx->heavy_slots, ctx->n_heavy, ctr_ints, bitmap_warps, a.cu_seqlens,
+                                        a.cu_seqlens_out, a.kept_idx, ctx->row_desc));
   return launch_merge_aggregate(ctx, a, s);
 }
 
@@ -535,15 +538,14 @@ int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
   if (heavy_blocks > ctx->sm_count) heavy_blocks = ctx->sm_count;
   const int blocks = light_blocks + heavy_blocks;
   if (a.dt == D3TOM_FP32)
-    aggregate_compact_kernel<float><<<blocks, kAggWarps * 32, 0, s>>>(
+    D3TOM_CUDA_TRY(ctx, launch_serialized(aggregate_compact_kernel<float>, blocks, kAggWarps * 32, 0, s,
         static_cast<const float*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out, a.B, a.D,
         chunks, a.total_out, heavy_blocks, mean, a.member_count, ctx->member_off, ctx->member_list, ctx->heavy_slots,
-        ctx->n_heavy, ctx->row_desc, static_cast<float*>(a.hidden_out), a.src_of_dst);
+        ctx->n_heavy, ctx->row_desc, static_cast<float*>(a.hidden_out), a.src_of_dst));
   else
-    aggregate_compact_kernel<__nv_bfloat16><<<blocks, kAggWarps * 32, 0, s>>>(
+    D3TOM_CUDA_TRY(ctx, launch_serialized(aggregate_compact_kernel<__nv_bfloat16>, blocks, kAggWarps * 32, 0, s,
         static_cast<const __nv_bfloat16*>(a.hidden), a.cu_seqlens, a.n_visual, a.kept_idx, a.cu_kept, a.cu_seqlens_out,
         a.B, a.D, chunks, a.total_out, heavy_blocks, mean, a.member_count, ctx->member_off, ctx->member_list,
-        ctx->heavy_slots, ctx->n_heavy, ctx->row_desc, static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst);
-  D3TOM_LAUNCH_CHECK(ctx);
+        ctx->heavy_slots, ctx->n_heavy, ctx->row_desc, static_cast<__nv_bfloat16*>(a.hidden_out), a.src_of_dst));
   return D3TOM_OK;
 }

@@ -49,7 +49,7 @@ struct StreamParams {
   const int4* row_desc;            // per output row: {source row, members or -1 (copy), list offset, request's first row}
   const int32_t* member_list;
   int32_t* src_of_dst;
-  int* work_counter;               // zero at launch
+  int* work_counter;               // [0] next work item, [1] CTAs done; both zero at launch, the last CTA zeroes them again
   int* dev_status;
   int total_out, D, col_splits, seg_bytes, slots, mean;
 };
@@ -73,6 +73,8 @@ aggregate_stream_kernel(StreamParams p) {
     abort_word = 0;
     ptx::fence_mbar_init();
   }
+  grid_dependency_wait();
+  grid_dependency_release();
   __syncthreads();
   const int seg_elems = p.seg_bytes / (int)sizeof(T);
   const long long n_items = (long long)p.total_out * p.col_splits;
@@ -136,6 +138,11 @@ aggregate_stream_kernel(StreamParams p) {
         header[s] = make_int4(-1, 0, 0, 0);
         ptx::mbar_arrive(&full[s]);
       }
+    }
+    // this CTA takes no more work; the last CTA to say so leaves both counters at zero for the next launch
+    if (lane == 0) {
+      __threadfence();
+      if (atomicAdd(p.work_counter + 1, 1) == (int)gridDim.x - 1) { p.work_counter[0] = 0; p.work_counter[1] = 0; }
     }
   } else {
     // ------------------------------------------------------------ consumer warps: 128 threads, 16 bytes per thread and pass
@@ -202,7 +209,6 @@ int launch_merge_aggregate_stream(d3tom_ctx* ctx, const MergeArgs& a, cudaStream
   p.src_of_dst = a.src_of_dst; p.work_counter = ctx->agg_counter; p.dev_status = ctx->dev_status;
   p.total_out = a.total_out; p.D = a.D; p.col_splits = splits; p.seg_bytes = (int)seg; p.slots = slots;
   p.mean = a.mode == D3TOM_AGG_MEAN ? 1 : 0;
-  D3TOM_CUDA_TRY(ctx, cudaMemsetAsync(ctx->agg_counter, 0, sizeof(int), s));
   const size_t smem = (size_t)slots * seg + 128;
   const long long items = (long long)a.total_out * splits;
   long long grid = 6LL * ctx->sm_count;                 // six CTAs fit one SM (32 KB of ring each): what limits the
@@ -210,11 +216,10 @@ int launch_merge_aggregate_stream(d3tom_ctx* ctx, const MergeArgs& a, cudaStream
   if (grid > items) grid = items;
   if (a.dt == D3TOM_FP32) {
     D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(aggregate_stream_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes + 128));
-    aggregate_stream_kernel<float><<<(int)grid, kStreamThreads, smem, s>>>(p);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(aggregate_stream_kernel<float>, (int)grid, kStreamThreads, smem, s, p));
   } else {
     D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(aggregate_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes + 128));
-    aggregate_stream_kernel<__nv_bfloat16><<<(int)grid, kStreamThreads, smem, s>>>(p);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(aggregate_stream_kernel<__nv_bfloat16>, (int)grid, kStreamThreads, smem, s, p));
   }
-  D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }

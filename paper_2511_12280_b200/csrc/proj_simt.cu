@@ -11,6 +11,7 @@ proj_simt_kernel(const T* __restrict__ x, const T* __restrict__ w, int n, int D,
                  T* __restrict__ q, T* __restrict__ k, T* __restrict__ v) {
   __shared__ float xs[32][33];
   __shared__ float ws[32][33];
+  grid_dependency_enter();
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int row = blockIdx.y * 32 + ty;       // token
   const int col = blockIdx.x * 32 + tx;       // output feature in [0, 3D)
@@ -36,13 +37,13 @@ int launch_proj_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* 
                      void* q, void* k, void* v, cudaStream_t s) {
   dim3 grid(ceil_div(3 * D, 32), ceil_div(total, 32));
   if (dt == D3TOM_FP32)
-    proj_simt_kernel<float><<<grid, 1024, 0, s>>>(static_cast<const float*>(x), static_cast<const float*>(w), total, D,
-                                                  static_cast<float*>(q), static_cast<float*>(k), static_cast<float*>(v));
+    D3TOM_CUDA_TRY(ctx, launch_serialized(proj_simt_kernel<float>, grid, 1024, 0, s, static_cast<const float*>(x),
+                                          static_cast<const float*>(w), total, D, static_cast<float*>(q),
+                                          static_cast<float*>(k), static_cast<float*>(v)));
   else
-    proj_simt_kernel<__nv_bfloat16><<<grid, 1024, 0, s>>>(static_cast<const __nv_bfloat16*>(x),
-                                                          static_cast<const __nv_bfloat16*>(w), total, D,
-                                                          static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k),
-                                                          static_cast<__nv_bfloat16*>(v));
-  D3TOM_LAUNCH_CHECK(ctx);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(proj_simt_kernel<__nv_bfloat16>, grid, 1024, 0, s,
+                                          static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w),
+                                          total, D, static_cast<__nv_bfloat16*>(q), static_cast<__nv_bfloat16*>(k),
+                                          static_cast<__nv_bfloat16*>(v)));
   return D3TOM_OK;
 }

@@ -29,6 +29,7 @@ select_kernel(const float* __restrict__ importance, const int32_t* __restrict__ 
               int32_t* __restrict__ kept_idx, uint8_t* __restrict__ keep_mask) {
   extern __shared__ uint32_t keys_s[];
   __shared__ SelectShared sh;
+  grid_dependency_enter();
   const int b = blockIdx.x;
   const int v0 = cu_vis[b], V = cu_vis[b + 1] - v0;
   const int k = keep_count[b];
@@ -154,9 +155,9 @@ int launch_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis
       D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
       attr_set = true;
     }
-    select_kernel<true><<<B, kThreads, smem, s>>>(importance, cu_vis, keep_count, cu_kept, kept_idx, keep_mask);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(select_kernel<true>, B, kThreads, smem, s, importance, cu_vis, keep_count, cu_kept, kept_idx, keep_mask));
   } else {
-    select_kernel<false><<<B, kThreads, 0, s>>>(importance, cu_vis, keep_count, cu_kept, kept_idx, keep_mask);
+    D3TOM_CUDA_TRY(ctx, launch_serialized(select_kernel<false>, B, kThreads, 0, s, importance, cu_vis, keep_count, cu_kept, kept_idx, keep_mask));
   }
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
