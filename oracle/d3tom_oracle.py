@@ -21,6 +21,8 @@ Readings of points the paper leaves open (each repeated where it is used):
   * aggregation: SUM is the paper's equation; MEAN divides by 1 + members.
   * kept tokens keep their original relative order in the output.
   * the schedule is indexed by decode order s = 0..T-1 (alpha grows with s).
+  * FFN_l is the gated form (three d x m matrices, as the 3ndm cost term
+    implies), without normalisation layers; the residual input is optional.
 
 Pins: every function here is pinned by tests/test_oracle_*.py (closed forms,
 brute force on tiny inputs, invariants, and the paper's printed FLOP tables
@@ -327,6 +329,51 @@ def post_layer(x, w_qkv, cu_seqlens, H, dtype="bf16"):
     q, k, v = proj_qkv(x, w_qkv, H, dtype)
     dh = q.shape[2]
     return round_storage(attention(q, k, v, cu_seqlens, 1.0 / np.sqrt(dh)), dtype)
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1, H <- FFN_l(H^): the rest of a Transformer block on the shortened
+# sequence.  The layer-cost equation of the FLOPs appendix counts 4 n d^2 for
+# the four d x d projections (Q, K, V and the attention output projection) and
+# 3 n d m for the feed-forward network, i.e. three d x m matrices.
+# Readings: the paper does not write the FFN out; three matrices of d x m are
+# the gated form, act = silu(x W_gate^T) * (x W_up^T), y = act W_down^T.  No
+# normalisation layer (its weights belong to a trained model); the residual
+# input is optional.
+# --------------------------------------------------------------------------
+def linear(x, w, residual=None, dtype="bf16"):
+    """y = residual + x W^T, rounded to the storage type.  w: [N, K], row o
+    holds the weights of output feature o.  With K = N = d this is the attention
+    output projection, the fourth d x d matrix of the 4 n d^2 term."""
+    y = np.asarray(x, np.float64) @ np.asarray(w, np.float64).T
+    if residual is not None:
+        y = y + np.asarray(residual, np.float64)
+    return round_storage(y, dtype)
+
+
+def silu(g):
+    """silu(g) = g * sigmoid(g) = g / (1 + exp(-g))."""
+    g = np.asarray(g, np.float64)
+    with np.errstate(over="ignore"):
+        return g / (1.0 + np.exp(-g))
+
+
+def ffn(x, w_gate_up, w_down, residual=None, dtype="bf16"):
+    """Gated feed-forward network, the 3 n d m term.  w_gate_up: [2m, d], rows
+    0..m-1 the gate matrix, rows m..2m-1 the up matrix; w_down: [d, m].
+    The activation act = silu(x W_gate^T) * (x W_up^T) is a stored tensor between
+    the two products and is rounded to the storage type; y = residual + act W_down^T,
+    rounded.  Returns (y, act)."""
+    x = np.asarray(x, np.float64)
+    w = np.asarray(w_gate_up, np.float64)
+    m = w.shape[0] // 2
+    gate = x @ w[:m].T
+    up = x @ w[m:].T
+    act = round_storage(silu(gate) * up, dtype)
+    y = act @ np.asarray(w_down, np.float64).T
+    if residual is not None:
+        y = y + np.asarray(residual, np.float64)
+    return round_storage(y, dtype), act
 
 
 # --------------------------------------------------------------------------

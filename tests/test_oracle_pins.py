@@ -413,3 +413,75 @@ def test_merge_kv_routing_depends_on_keys_only_and_conserves_mass():
     # keeping everything is the identity on both caches
     ident = orc.merge_kv(K, Va, [0, V + P], [V], [np.arange(V)], orc.SUM, "fp32")
     assert np.array_equal(ident["k_out"], K) and np.array_equal(ident["v_out"], Va)
+
+
+# ------------------------------------------------------------------ rest of the block (Algorithm 1, FFN_l; layer-cost equation)
+def test_linear_row_o_of_w_holds_output_feature_o_and_the_residual_is_added():
+    w = np.array([[1.0, 2.0], [3.0, 4.0], [0.5, -1.0]])
+    x = np.array([[1.0, 10.0], [0.0, 1.0]])
+    y = orc.linear(x, w, dtype="fp32")
+    assert np.array_equal(y, np.array([[21.0, 43.0, -9.5], [2.0, 4.0, -1.0]]))
+    res = np.array([[1.0, 1.0, 1.0], [0.0, 0.0, 0.25]])
+    assert np.array_equal(orc.linear(x, w, res, dtype="fp32"), y + res)
+    # identity weights: the result is the storage rounding of x + residual
+    r = rng(40)
+    xb = orc.round_bf16(r.standard_normal((5, 8)))
+    rb = orc.round_bf16(r.standard_normal((5, 8)))
+    assert np.array_equal(orc.linear(xb, np.eye(8), rb, dtype="bf16"), orc.round_bf16(xb + rb))
+
+
+def test_silu_closed_forms():
+    # sigmoid(ln 3) = 3/4
+    assert abs(orc.silu(math.log(3.0)) - 0.75 * math.log(3.0)) < 1e-15
+    assert orc.silu(0.0) == 0.0
+    assert abs(orc.silu(50.0) - 50.0) < 1e-12 and abs(orc.silu(-50.0)) < 1e-12
+    assert orc.silu(-1000.0) == 0.0          # exp overflows to inf, the quotient is -0
+    g = rng(41).standard_normal(1000) * 4
+    want = torch.nn.functional.silu(torch.from_numpy(g)).numpy()
+    assert np.allclose(orc.silu(g), want, rtol=1e-13, atol=1e-15)
+
+
+def test_ffn_gate_and_up_are_not_interchangeable_closed_form():
+    # one token, d = 1, m = 1: gate pre-activation ln 3, up 2, down 1 -> 0.75 ln3 * 2
+    y, act = orc.ffn(np.array([[1.0]]), np.array([[math.log(3.0)], [2.0]]), np.array([[1.0]]), dtype="fp32")
+    assert abs(y[0, 0] - 1.5 * math.log(3.0)) < 1e-6 and abs(act[0, 0] - 1.5 * math.log(3.0)) < 1e-6
+    # zero gate matrix: silu(0) = 0, the block returns its residual
+    r = rng(42)
+    x = r.standard_normal((4, 6)); res = orc.round_bf16(r.standard_normal((4, 6)))
+    w = np.concatenate([np.zeros((10, 6)), r.standard_normal((10, 6))])
+    y, act = orc.ffn(x, w, r.standard_normal((6, 10)), res, dtype="bf16")
+    assert np.array_equal(act, np.zeros((4, 10))) and np.array_equal(y, res)
+
+
+def test_ffn_equals_pure_python_brute_force_and_torch_fp64():
+    r = rng(43)
+    n, d, m = 3, 5, 7
+    x = r.standard_normal((n, d)); wgu = r.standard_normal((2 * m, d)) * 0.5
+    wd = r.standard_normal((d, m)) * 0.5; res = r.standard_normal((n, d))
+    want = np.zeros((n, d))
+    for i in range(n):
+        act = []
+        for j in range(m):
+            g = sum(x[i, c] * wgu[j, c] for c in range(d))
+            u = sum(x[i, c] * wgu[m + j, c] for c in range(d))
+            act.append(g / (1.0 + math.exp(-g)) * u)
+        for o in range(d):
+            want[i, o] = res[i, o] + sum(act[j] * wd[o, j] for j in range(m))
+    y, _ = orc.ffn(x, wgu, wd, res, dtype="fp32")
+    assert np.allclose(y, want, rtol=1e-6, atol=1e-6)      # fp32 storage rounding only
+    F = torch.nn.functional
+    tx, tw, td = torch.from_numpy(x), torch.from_numpy(wgu), torch.from_numpy(wd)
+    t = F.linear(F.silu(F.linear(tx, tw[:m])) * F.linear(tx, tw[m:]), td) + torch.from_numpy(res)
+    assert np.allclose(y, t.numpy(), rtol=1e-6, atol=1e-6)
+
+
+def test_ffn_activation_is_rounded_to_storage_before_the_second_product():
+    r = rng(44)
+    n, d, m = 4, 8, 8
+    x = orc.round_bf16(r.standard_normal((n, d)))
+    wgu = orc.round_bf16(r.standard_normal((2 * m, d)) * 0.5)
+    y, act = orc.ffn(x, wgu, np.eye(m), dtype="bf16")       # identity down projection: y is the activation
+    assert np.array_equal(act, orc.round_bf16(act))
+    assert np.array_equal(y, act)
+    exact = orc.silu(x @ wgu[:m].T) * (x @ wgu[m:].T)
+    assert np.array_equal(act, orc.round_bf16(exact)) and not np.array_equal(act, exact)
