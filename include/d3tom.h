@@ -12,6 +12,8 @@
  *   d3tom_attn_varlen       bidirectional attention over the shortened sequences
  *   d3tom_merge_kv          the same routing applied to a cached K/V prefix
  *   d3tom_proj_qkv          (supporting) Q,K,V projection of a post-merge layer
+ *   d3tom_linear, d3tom_ffn (supporting) output projection and gated feed-forward
+ *                           network of a post-merge block
  *
  * Conventions shared by every call
  * --------------------------------
@@ -247,6 +249,33 @@ int d3tom_attn_varlen(d3tom_ctx* ctx, d3tom_dtype dt,
  * q, k, v [total, D] out, fp32 accumulation, one rounding to the storage type. */
 int d3tom_proj_qkv(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_qkv,
                    int total, int D, void* q, void* k, void* v, d3tom_stream stream);
+
+/* Algorithm 1, H <- FFN_l(H^), and the layer-cost equation of the FLOPs appendix
+ * (4 n d^2 for four d x d projections, 3 n d m for the feed-forward network): the
+ * rest of a Transformer block, run on the shortened sequence after the merge.
+ * The paper does not write the block out; this library takes the gated form the
+ * three d x m matrices imply and no normalisation layers.
+ *
+ * d3tom_linear: out = residual + x w^T, fp32 accumulation, one rounding to the
+ * storage type.  x [rows, K]; w [N, K] row-major, row o holds the weights of
+ * output feature o; residual [rows, N] or NULL; out [rows, N].  With K = N = D
+ * this is the attention output projection.  out may be the residual buffer itself
+ * (in-place add) but not x.  All pointers are device memory, caller-owned.
+ * bf16 on the tensor-core path needs K % 64 == 0 and N % 128 == 0
+ * (D3TOM_ERR_UNSUPPORTED otherwise); fp32 has no such limit. */
+int d3tom_linear(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w, const void* residual,
+                 int rows, int K, int N, void* out, d3tom_stream stream);
+
+/* d3tom_ffn: act = silu(x Wg^T) * (x Wu^T), rounded to the storage type, then
+ * out = residual + act Wd^T.  x [rows, D]; w_gate_up [2m, D]: rows 0..m-1 are
+ * Wg, rows m..2m-1 are Wu; w_down [D, m]; residual [rows, D] or NULL;
+ * act [rows, m] is scratch the caller provides (device memory; holds the
+ * activation afterwards); out [rows, D], may be the residual buffer.  Two kernel
+ * launches: the gate and up products share one pass whose epilogue applies
+ * silu(gate) * up, so neither product is written out.  bf16 on the tensor-core
+ * path needs D % 128 == 0 and m % 128 == 0. */
+int d3tom_ffn(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_gate_up, const void* w_down,
+              const void* residual, int rows, int D, int m, void* act, void* out, d3tom_stream stream);
 
 #ifdef __cplusplus
 }

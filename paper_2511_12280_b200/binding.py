@@ -55,6 +55,8 @@ _SIGNATURES = {
     "d3tom_merge_kv": (_I, [_P, _I, _I, _P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P, _P, _P]),
     "d3tom_attn_varlen": (_I, [_P, _I, _P, _P, _P, _P, _I, _I, _I, _F, _P, _P]),
     "d3tom_proj_qkv": (_I, [_P, _I, _P, _P, _I, _I, _P, _P, _P, _P]),
+    "d3tom_linear": (_I, [_P, _I, _P, _P, _P, _I, _I, _I, _P, _P]),
+    "d3tom_ffn": (_I, [_P, _I, _P, _P, _P, _P, _I, _I, _I, _P, _P, _P]),
 }
 
 
@@ -202,3 +204,12 @@ class Context:
     def d3tom_proj_qkv(self, x, w_qkv, total, D, q, k, v, stream=None):
         _check(load().d3tom_proj_qkv(self._h, _dt(x), _ptr(x), _ptr(w_qkv), total, D, _ptr(q), _ptr(k), _ptr(v),
                                      _stream(stream)), "d3tom_proj_qkv")
+
+    def d3tom_linear(self, x, w, residual, rows, K, N, out, stream=None):
+        _check(load().d3tom_linear(self._h, _dt(x), _ptr(x), _ptr(w), _ptr(residual) if residual is not None else None,
+                                   rows, K, N, _ptr(out), _stream(stream)), "d3tom_linear")
+
+    def d3tom_ffn(self, x, w_gate_up, w_down, residual, rows, D, m, act, out, stream=None):
+        _check(load().d3tom_ffn(self._h, _dt(x), _ptr(x), _ptr(w_gate_up), _ptr(w_down),
+                                _ptr(residual) if residual is not None else None, rows, D, m, _ptr(act), _ptr(out),
+                                _stream(stream)), "d3tom_ffn")

@@ -311,4 +311,40 @@ int d3tom_proj_qkv(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_
   return launch_proj_simt(ctx, dt, x, w_qkv, total, D, q, k, v, s);
 }
 
+int d3tom_linear(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w, const void* residual, int rows, int K,
+                 int N, void* out, d3tom_stream stream) {
+  if (ctx == nullptr) return D3TOM_ERR_INVALID_ARG;
+  if (dt != D3TOM_FP32 && dt != D3TOM_BF16) return D3TOM_ERR_UNSUPPORTED;
+  if (x == nullptr || w == nullptr || out == nullptr || rows < 0 || K <= 0 || N <= 0 || x == out)
+    return D3TOM_ERR_INVALID_ARG;
+  if (rows == 0) return D3TOM_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return D3TOM_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == D3TOM_BF16 && !ctx->reference_kernels) return launch_linear_tc(ctx, x, w, residual, rows, K, N, out, s);
+  return launch_linear_simt(ctx, dt, x, w, residual, rows, K, N, out, s);
+}
+
+int d3tom_ffn(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_gate_up, const void* w_down,
+              const void* residual, int rows, int D, int m, void* act, void* out, d3tom_stream stream) {
+  if (ctx == nullptr) return D3TOM_ERR_INVALID_ARG;
+  if (dt != D3TOM_FP32 && dt != D3TOM_BF16) return D3TOM_ERR_UNSUPPORTED;
+  if (x == nullptr || w_gate_up == nullptr || w_down == nullptr || act == nullptr || out == nullptr || rows < 0 ||
+      D <= 0 || m <= 0 || act == out || act == x || act == residual)
+    return D3TOM_ERR_INVALID_ARG;
+  if (rows == 0) return D3TOM_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return D3TOM_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dt == D3TOM_BF16 && !ctx->reference_kernels) {
+    if (D % 128 != 0 || m % 128 != 0) return D3TOM_ERR_UNSUPPORTED;   // checked before anything is launched
+    const int st = launch_gate_up_tc(ctx, x, w_gate_up, rows, D, m, act, s);
+    if (st != D3TOM_OK) return st;
+    return launch_linear_tc(ctx, act, w_down, residual, rows, m, D, out, s);
+  }
+  const int st = launch_gate_up_simt(ctx, dt, x, w_gate_up, rows, D, m, act, s);
+  if (st != D3TOM_OK) return st;
+  return launch_linear_simt(ctx, dt, act, w_down, residual, rows, m, D, out, s);
+}
+
 }  // extern "C"

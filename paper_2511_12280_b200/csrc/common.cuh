@@ -181,3 +181,12 @@ int launch_proj_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* 
                      void* q, void* k, void* v, cudaStream_t s);
 int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int D,
                    void* q, void* k, void* v, cudaStream_t s);
+// y = residual + x w^T and act = silu(x Wg^T) * (x Wu^T): the rest of a block (output projection, feed-forward network)
+int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* residual, int rows, int K, int N,
+                     void* out, cudaStream_t s);
+int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int rows, int D, int m, void* act,
+                      cudaStream_t s);
+int launch_linear_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w, const void* residual, int rows,
+                       int K, int N, void* out, cudaStream_t s);
+int launch_gate_up_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w_gate_up, int rows, int D, int m,
+                        void* act, cudaStream_t s);

@@ -1,5 +1,5 @@
 // bf16 x bf16 -> fp32 "NT" GEMM on tcgen05 tensor cores, C[m, n] = sum_k A[m, k] B[n, k],
-// with two fused epilogues:
+// with four fused epilogues:
 //
 //   kEpiProj  the Q,K,V projection of a post-merge layer (Sec. 3.2.1, Q = H W_Q,
 //             K = H W_K): rounds to bf16 and writes the tile into q, k or v.
@@ -7,6 +7,12 @@
 //             over the kept set): scales the dot products by the two inverse norms
 //             and folds every pruned row's candidates into its packed 64-bit
 //             running maximum, so the (V x k) similarity matrix never reaches HBM.
+//   kEpiLinear  y = residual + x W^T rounded to bf16: the attention output projection and the
+//             down projection of the feed-forward network (Algorithm 1, FFN_l; the fourth
+//             d x d matrix of the 4nd^2 term and the third d x m matrix of the 3ndm term).
+//   kEpiGateUp  the first two d x m matrices of the feed-forward network in one pass: a 256-wide
+//             tile is 128 gate rows and the 128 up rows of the same features, and the epilogue
+//             writes act = silu(gate) * up, so neither product reaches HBM.
 //
 // Persistent CTAs (one per SM) walk over the 128 x BN output tiles, M fastest so that the
 // BN x K operand stays hot in L2 while the M tiles that share it are computed.  Warps 0
@@ -22,7 +28,7 @@ namespace {
 constexpr int kBM = 128, kBK = 64;
 constexpr int kGemmThreads = 224;      // warps: 0 A loads, 1 MMA, 2..5 epilogue, 6 B loads
 
-enum { kEpiProj = 0, kEpiSim = 1 };
+enum { kEpiProj = 0, kEpiSim = 1, kEpiLinear = 2, kEpiGateUp = 3 };
 constexpr int kMaxKSplits = 4;        // K slices per similarity tile at most
 
 struct GemmParams {
@@ -35,6 +41,11 @@ struct GemmParams {
   __nv_bfloat16* out[3];      // q, k, v
   int out_rows;               // total tokens
   int out_cols;               // D
+  // linear / gate-up: rows are out_rows
+  __nv_bfloat16* lin_out;     // [out_rows, ld_out]
+  const __nv_bfloat16* residual;   // [out_rows, ld_out] or null (linear only; may be lin_out itself)
+  int ld_out;                 // N of the linear layer; m for the gate-up pass
+  int up_row_offset;          // gate-up: row of the weight matrix where the up matrix starts (m)
   // similarity
   const int32_t* cu_seqlens; const int32_t* cu_vis; const int32_t* cu_kept; const int32_t* assign;
   const float* inv_norm; const float* inv_norm_kept;
@@ -75,7 +86,8 @@ struct TileCoord {
     const int rest = t / p.m_tiles;
     ni = rest % p.n_tiles;
     b = rest / p.n_tiles;
-    m0 = mi * kBM; n0 = ni * BN; a_row = m0; b_row = n0;
+    // (a gate-up tile covers BN / 2 output features: its B rows are 128 gate rows and 128 up rows)
+    m0 = mi * kBM; n0 = ni * (EPI == kEpiGateUp ? BN / 2 : BN); a_row = m0; b_row = n0;
     Vb = kb = v0 = k0 = 0;
     if (EPI == kEpiSim) {
       v0 = p.cu_vis[b]; Vb = p.cu_vis[b + 1] - v0;
@@ -165,7 +177,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           ok = ptx::mbar_wait(&empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.dev_status);
           if (!ok) break;
           ptx::mbar_arrive_expect_tx(&full[s], stage_bytes);
-          ptx::tma_load_2d(ring + s * stage_bytes, tm, &full[s], kbk * kBK, row0);
+          if (EPI == kEpiGateUp && !is_a) {        // two boxes of BN / 2 rows: gate rows, then the up rows of the same features
+            ptx::tma_load_2d(ring + s * stage_bytes, tm, &full[s], kbk * kBK, row0);
+            ptx::tma_load_2d(ring + s * stage_bytes + stage_bytes / 2, tm, &full[s], kbk * kBK, p.up_row_offset + row0);
+          } else {
+            ptx::tma_load_2d(ring + s * stage_bytes, tm, &full[s], kbk * kBK, row0);
+          }
         }
       }
     }
@@ -244,6 +261,59 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 w[j] = *reinterpret_cast<uint32_t*>(&h2);
               }
               *reinterpret_cast<uint4*>(dst + c + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else if (EPI == kEpiLinear) {
+        const int grow = tc.m0 + row;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_row + c, r);
+          ptx::tmem_wait_ld();
+          if (grow < p.out_rows) {
+            const size_t off = (size_t)grow * p.ld_out + tc.n0 + c;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4] = {0u, 0u, 0u, 0u};
+              if (p.residual != nullptr) {
+                const uint4 rr = *reinterpret_cast<const uint4*>(p.residual + off + i);
+                w[0] = rr.x; w[1] = rr.y; w[2] = rr.z; w[3] = rr.w;
+              }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float lo = __uint_as_float(r[i + 2 * j]) + __uint_as_float(w[j] << 16);
+                const float hi = __uint_as_float(r[i + 2 * j + 1]) + __uint_as_float(w[j] & 0xffff0000u);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+                w[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(p.lin_out + off + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else if (EPI == kEpiGateUp) {
+        const int grow = tc.m0 + row;
+#pragma unroll 1
+        for (int c = 0; c < BN / 2; c += 32) {
+          uint32_t g[32], u[32];
+          ptx::tmem_ld32(t_row + c, g);
+          ptx::tmem_ld32(t_row + BN / 2 + c, u);
+          ptx::tmem_wait_ld();
+          if (grow < p.out_rows) {
+            __nv_bfloat16* dst = p.lin_out + (size_t)grow * p.ld_out + tc.n0 + c;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float g0 = __uint_as_float(g[i + 2 * j]), g1 = __uint_as_float(g[i + 2 * j + 1]);
+                // silu(g) = g / (1 + exp(-g)); for very negative g the divisor is inf and the quotient 0
+                const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[i + 2 * j]);
+                const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[i + 2 * j + 1]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
+                w[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
         }
@@ -419,6 +489,50 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
   if (bn == 256) return launch_gemm<256, kEpiProj>(ctx, ta, tb, p, s);
   if (bn == 192) return launch_gemm<192, kEpiProj>(ctx, ta, tb, p, s);
   return launch_gemm<128, kEpiProj>(ctx, ta, tb, p, s);
+}
+
+int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* residual, int rows, int K, int N,
+                     void* out, cudaStream_t s) {
+  if (K % kBK != 0 || N % 128 != 0) return D3TOM_ERR_UNSUPPORTED;
+  CUtensorMap ta, tb;
+  int r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)K, (uint64_t)K, kBM);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  GemmParams p = {};
+  p.num_k_blocks = K / kBK;
+  p.lin_out = static_cast<__nv_bfloat16*>(out); p.residual = static_cast<const __nv_bfloat16*>(residual);
+  p.ld_out = N; p.out_rows = rows; p.dev_status = ctx->dev_status;
+  p.m_tiles = ceil_div(rows, kBM); p.batch = 1; p.k_splits = 1;
+  // tile width as for the Q,K,V projection: fewest rounds of tiles over the SMs, weighted by the cycles per k-block
+  int bn = 128;
+  double best_cost = 1e30;
+  for (int cand : {256, 192, 128}) {
+    if (N % cand != 0) continue;
+    const long long tiles = (long long)p.m_tiles * (N / cand);
+    const double rounds = (double)((tiles + ctx->sm_count - 1) / ctx->sm_count);
+    const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
+    if (cost < best_cost) { best_cost = cost; bn = cand; }
+  }
+  r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  p.n_tiles = N / bn;
+  if (bn == 256) return launch_gemm<256, kEpiLinear>(ctx, ta, tb, p, s);
+  if (bn == 192) return launch_gemm<192, kEpiLinear>(ctx, ta, tb, p, s);
+  return launch_gemm<128, kEpiLinear>(ctx, ta, tb, p, s);
+}
+
+int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int rows, int D, int m, void* act,
+                      cudaStream_t s) {
+  if (D % kBK != 0 || m % 128 != 0) return D3TOM_ERR_UNSUPPORTED;
+  CUtensorMap ta, tb;
+  int r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)D, (uint64_t)D, kBM);
+  if (r == 0) r = make_tmap_bf16_2d(&tb, w_gate_up, (uint64_t)2 * m, (uint64_t)D, (uint64_t)D, 128);
+  if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+  GemmParams p = {};
+  p.num_k_blocks = D / kBK;
+  p.lin_out = static_cast<__nv_bfloat16*>(act); p.ld_out = m; p.up_row_offset = m; p.out_rows = rows;
+  p.dev_status = ctx->dev_status;
+  p.m_tiles = ceil_div(rows, kBM); p.n_tiles = m / 128; p.batch = 1; p.k_splits = 1;
+  return launch_gemm<256, kEpiGateUp>(ctx, ta, tb, p, s);
 }
 
 int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {

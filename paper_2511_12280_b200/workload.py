@@ -26,6 +26,8 @@ this order):
      extra mass on the salient keys);
   5. everything is rounded to the storage type (bf16 or fp32);
   6. post-merge layer weights W^l ~ N(0, 0.02), [3D, D], drawn last.
+``block_inputs`` draws the tensors of the rest of a block (output projection,
+feed-forward network) from a generator of its own.
 """
 from __future__ import annotations
 
@@ -154,6 +156,17 @@ def make_workload(name, dtype, H, dh, seed, n_clusters, requests, post_layers=0,
         keep_ratio=[float(r["r"]) for r in requests], decider_pos=decs, salient=sals,
         q_base=torch.cat(qs), k=torch.cat(ks), v=torch.cat(vs), u=us, w_post=w_post,
         T=T, decode_order=decode_order, mean_keep_ratio=mean_keep_ratio)
+
+
+def block_inputs(seed: int, rows: int, D: int, m: int, dtype: str = "bf16"):
+    """Inputs for the rest of a post-merge block (output projection + gated feed-forward network) at LLaDA-8B
+    shapes (D = 4096, m = 12288) or smaller: x, residual ~ N(0,1) [rows, D]; W_o [D, D], W_gate_up [2m, D],
+    W_down [D, m] ~ N(0, 0.02), one generator, drawn in this order, rounded to the storage type."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    draw = lambda shape, sigma: torch.from_numpy(_normal(rng, shape, sigma)).to(tdt)
+    return dict(x=draw((rows, D), 1.0), residual=draw((rows, D), 1.0), w_o=draw((D, D), WEIGHT_SIGMA),
+                w_gate_up=draw((2 * m, D), WEIGHT_SIGMA), w_down=draw((D, m), WEIGHT_SIGMA))
 
 
 def config(name: str) -> Workload:

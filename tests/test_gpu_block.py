@@ -1,0 +1,129 @@
+"""d3tom_linear and d3tom_ffn (Algorithm 1, FFN_l: the rest of a post-merge block) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import d3tom_oracle as orc
+from paper_2511_12280_b200 import binding as B_
+from paper_2511_12280_b200 import workload as wl
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def make_ctx(rows, dtype):
+    # the dense layers use no scratch of the context; head geometry only has to be valid
+    return B_.Context(max(rows, 1), 1, 2, 64 if dtype == "bf16" else 8, 1, 1)
+
+
+def run_linear(rows, K, N, dtype, residual, in_place=False, seed=0):
+    dev = torch.device("cuda", 0)
+    t = wl.block_inputs(seed, rows, max(K, N), 8, dtype)
+    x = t["x"][:, :K].contiguous()
+    w = t["w_o"][:N, :K].contiguous() * 4           # keeps outputs O(1) at small K
+    res = t["residual"][:, :N].contiguous() if residual else None
+    ctx = make_ctx(rows, dtype)
+    xd, wd = x.to(dev), w.to(dev)
+    if in_place:
+        out = res.to(dev); resd = out
+    else:
+        out = torch.full((rows, N), float("nan"), dtype=x.dtype, device=dev)
+        resd = res.to(dev) if residual else None
+    ctx.d3tom_linear(xd, wd, resd, rows, K, N, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    want = orc.linear(pu.f64(x), pu.f64(w), pu.f64(res) if residual else None, dtype)
+    pu.assert_close(pu.f64(out), want, dtype, "linear %dx%dx%d" % (rows, K, N))
+    ctx.close()
+
+
+@pytest.mark.parametrize("N", [128, 384, 512, 768])      # tile widths 128, 192 / 128, 256, 256 / 192
+def test_linear_bf16_every_tile_width_ragged_rows(N):
+    run_linear(300, 256, N, "bf16", residual=True)
+
+
+def test_linear_bf16_without_residual_and_in_place():
+    run_linear(300, 192, 256, "bf16", residual=False)
+    run_linear(129, 320, 256, "bf16", residual=True, in_place=True)
+    run_linear(1, 64, 128, "bf16", residual=True)
+
+
+def test_linear_fp32_odd_sizes():
+    run_linear(70, 50, 45, "fp32", residual=True)
+    run_linear(33, 7, 3, "fp32", residual=False)
+
+
+def run_ffn(rows, D, m, dtype, residual=True, seed=1, sample_rows=None):
+    dev = torch.device("cuda", 0)
+    t = wl.block_inputs(seed, rows, D, m, dtype)
+    scale = 4.0 if D < 1024 else 1.0                  # keeps gate pre-activations O(1) at small D
+    x, wgu, wdn = t["x"], t["w_gate_up"] * scale, t["w_down"] * scale
+    res = t["residual"] if residual else None
+    ctx = make_ctx(rows, dtype)
+    act = torch.full((rows, m), float("nan"), dtype=x.dtype, device=dev)
+    out = torch.full((rows, D), float("nan"), dtype=x.dtype, device=dev)
+    ctx.d3tom_ffn(x.to(dev), wgu.to(dev), wdn.to(dev), res.to(dev) if residual else None, rows, D, m, act, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    sel = np.arange(rows) if sample_rows is None else np.asarray(sample_rows)
+    xs, rs = pu.f64(x)[sel], (pu.f64(res)[sel] if residual else None)
+    want_out, want_act = orc.ffn(xs, pu.f64(wgu), pu.f64(wdn), rs, dtype)
+    act_g, out_g = pu.f64(act)[sel], pu.f64(out)[sel]
+    pu.assert_close(act_g, want_act, dtype, "ffn activation")
+    # second product fed the GPU's own activation (a bf16 rounding flip in act cannot cascade), then free-running
+    pu.assert_close(out_g, orc.linear(act_g, pu.f64(wdn), rs, dtype), dtype, "ffn output, teacher-forced")
+    pu.assert_close(out_g, want_out, dtype, "ffn output")
+    if sample_rows is not None:
+        assert torch.isfinite(out.float()).all() and torch.isfinite(act.float()).all()
+    ctx.close()
+
+
+def test_ffn_bf16_ragged_rows_several_tiles():
+    run_ffn(300, 256, 384, "bf16")
+    run_ffn(127, 128, 128, "bf16", residual=False)
+
+
+def test_ffn_fp32_odd_sizes():
+    run_ffn(37, 24, 20, "fp32")
+
+
+def test_ffn_bf16_llada_shape_sampled_rows():
+    # rows of the shortened sequence of the 4096-visual-token configuration, d = 4096, m = 12288;
+    # the oracle computes a sample of rows (the layers act row by row)
+    run_ffn(1216, 4096, 12288, "bf16", sample_rows=[0, 1, 127, 128, 640, 1151, 1152, 1215])
+
+
+def test_linear_bf16_llada_shape_sampled_rows():
+    dev = torch.device("cuda", 0)
+    rows, D = 1216, 4096
+    t = wl.block_inputs(2, rows, D, 8, "bf16")
+    ctx = make_ctx(rows, "bf16")
+    out = torch.full((rows, D), float("nan"), dtype=torch.bfloat16, device=dev)
+    ctx.d3tom_linear(t["x"].to(dev), t["w_o"].to(dev), t["residual"].to(dev), rows, D, D, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0 and torch.isfinite(out.float()).all()
+    sel = np.array([0, 127, 128, 1000, 1215])
+    want = orc.linear(pu.f64(t["x"])[sel], pu.f64(t["w_o"]), pu.f64(t["residual"])[sel], "bf16")
+    pu.assert_close(pu.f64(out)[sel], want, "bf16", "output projection")
+    ctx.close()
+
+
+def test_unsupported_shapes_and_bad_arguments_are_refused_on_the_host():
+    dev = torch.device("cuda", 0)
+    ctx = make_ctx(64, "bf16")
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device=dev)
+    lib = B_.load()
+    with pytest.raises(RuntimeError, match="UNSUPPORTED|unsupported"):
+        ctx.d3tom_linear(z(64, 64), z(100, 64), None, 64, 64, 100, z(64, 100))       # N not a multiple of 128
+    with pytest.raises(RuntimeError, match="UNSUPPORTED|unsupported"):
+        ctx.d3tom_linear(z(64, 40), z(128, 40), None, 64, 40, 128, z(64, 128))        # K not a multiple of 64
+    with pytest.raises(RuntimeError, match="UNSUPPORTED|unsupported"):
+        ctx.d3tom_ffn(z(64, 128), z(200, 128), z(128, 100), None, 64, 128, 100, z(64, 100), z(64, 128))
+    x = z(64, 128)
+    with pytest.raises(RuntimeError, match="INVALID|invalid"):
+        ctx.d3tom_linear(x, z(128, 128), None, 64, 128, 128, x)                       # out must not be x
+    ctx.d3tom_linear(x, z(128, 128), None, 0, 128, 128, z(64, 128))                  # no rows: nothing to do
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ctx.close()
