@@ -188,6 +188,49 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
+def block_timings(step, w, w_post0, q, k, v, dev, timed, reps):
+    """The rest of a post-merge block (Algorithm 1, FFN_l; layer-cost equation of the FLOPs appendix): output
+    projection and gated feed-forward network at the shortened length N_m, and the whole block at N_m and at the
+    full length N, so that the measured saving of a post-merge layer can be set beside the FLOPs ratio.
+    m = 3 d (12288 at d = 4096, the LLaDA-8B width)."""
+    import torch
+    from paper_2511_12280_b200 import workload as wl
+    timed_cold = timed
+
+    def timed(fn, iters):            # one untimed call first: these kernels have not run yet
+        fn()
+        return timed_cold(fn, iters)
+    D, m = step.D, 3 * step.D
+    t = wl.block_inputs(1000, 8, D, m, w.dtype)           # weights only; the rows come from the step's own tensors
+    w_o, w_gu, w_dn = t["w_o"].to(dev), t["w_gate_up"].to(dev), t["w_down"].to(dev)
+    ctx = step.ctx
+    out = {}
+    n_full, n_m = step.total, step.total_out
+    act = torch.empty(n_full, m, dtype=q.dtype, device=dev)
+    y = torch.empty(n_full, D, dtype=q.dtype, device=dev)
+    z = torch.empty(n_full, D, dtype=q.dtype, device=dev)
+    q3, k3, v3 = (torch.empty(n_full, D, dtype=q.dtype, device=dev) for _ in range(3))
+    x_m, x_full = step.hidden_out, step.attn_out
+    for tag, n, x, cu, mx in (("Nm", n_m, x_m, step.cu_out, step.max_out), ("N", n_full, x_full, step.cu_seqlens, step.max_seqlen)):
+        parts = {
+            "proj_qkv": timed(lambda: ctx.d3tom_proj_qkv(x, w_post0, n, D, q3, k3, v3), reps),
+            "attn": timed(lambda: ctx.d3tom_attn_varlen(q3, k3, v3, cu, step.nB, n, mx, step.scale, y), reps),
+            "proj_out": timed(lambda: ctx.d3tom_linear(y, w_o, x, n, D, D, z), reps),
+            "ffn": timed(lambda: ctx.d3tom_ffn(z, w_gu, w_dn, z, n, D, m, act, y), reps),
+        }
+        parts["block"] = sum(parts.values())
+        out[tag] = parts
+    lens_m, lens_f = step.out_lens_h, step.seqlens_h
+    macs = lambda lens: sum(4.0 * n * D * D + 2.0 * n * n * D + 3.0 * n * D * m for n in lens)      # layer-cost equation
+    out["proj_out_tflops_Nm"] = 2.0 * n_m * D * D / (out["Nm"]["proj_out"] * 1e-6) / 1e12
+    out["ffn_tflops_Nm"] = 6.0 * n_m * D * m / (out["Nm"]["ffn"] * 1e-6) / 1e12
+    out["ffn_tflops_N"] = 6.0 * n_full * D * m / (out["N"]["ffn"] * 1e-6) / 1e12
+    out["layer_time_ratio_Nm_over_N"] = out["Nm"]["block"] / out["N"]["block"]
+    out["layer_flops_ratio_Nm_over_N"] = macs(lens_m) / macs(lens_f)
+    out["m"] = m
+    return out
+
+
 def make_kv_cache_case(step, w, k, v, dev):
     """Returns a callable that runs d3tom_merge_kv on the K/V rows of every request's [visual | prompt]
     prefix with the kept set that the step's select produced."""
@@ -222,6 +265,7 @@ def main():
     ap.add_argument("--config", default="C2", choices=sorted(WORKLOAD_TEXT))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-block", action="store_true", help="skip the timing of the rest of a post-merge block")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
     ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "step"],
                     help="profiling aid: after one full step, run just this call --steps times and exit")
@@ -402,6 +446,12 @@ def main():
         # the same routing applied to the cached K/V prefix (Sec. 4.4): caches = K, V rows of [visual | prompt]
         kv = make_kv_cache_case(step, w, k, v, dev)
         br["merge_kv"] = timed(kv, reps)
+        # the rest of a post-merge block at N_m and at N (tensor-core path: bf16, widths in multiples of 128)
+        block = None
+        if step.n_post and w.dtype == "bf16" and step.D % 128 == 0 and not args.no_block:
+            block = block_timings(step, w, w_post[0], q, k, v, dev, timed, max(5, reps // 4))
+            br["proj_out"] = block["Nm"]["proj_out"]
+            br["ffn"] = block["Nm"]["ffn"]
         # the dominant kernel alone (no importance side-work): the attention kernel at the merge-layer length
         attn_kernel_us = timed(lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
                                                                   step.max_seqlen, step.scale, step.attn_out), reps)
@@ -482,6 +532,8 @@ def main():
         "peaks": dict(peaks, kind=peak_kind),
     }
 
+    if block is not None:
+        line["block"] = block
     if per_step is not None:
         line["per_step_us"] = per_step
         line["trajectory_total_us"] = float(sum(per_step))

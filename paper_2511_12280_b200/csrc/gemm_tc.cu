@@ -34,8 +34,9 @@ constexpr int kMaxKSplits = 4;        // K slices per similarity tile at most
 struct GemmParams {
   int num_k_blocks;           // K / 64
   int m_tiles, n_tiles, batch;   // tile grid (per request for the similarity); tiles outside a request are skipped
-  int k_splits;               // similarity with few tiles: each tile's K range is cut into this many work units
-  float* split_ws;            // [tiles * k_splits][BN][128] fp32 partial tiles (column-major: coalesced per warp)
+  int k_splits;               // tiles from `full_tiles` on have their K range cut into this many work units
+  int full_tiles;             // the first tiles of the walk are whole work units (0: every tile is cut)
+  float* split_ws;            // [(tiles - full_tiles) * k_splits][BN][128] fp32 partial tiles (column-major: coalesced per warp)
   int* split_counters;        // [tiles] parts done; zero between launches
   // projection
   __nv_bfloat16* out[3];      // q, k, v
@@ -51,6 +52,17 @@ struct GemmParams {
   const float* inv_norm; const float* inv_norm_kept;
   unsigned long long* best; float* sim_debug; int max_kept;
   int* dev_status;
+};
+
+// Work unit u of the walk: tile t, K slice sp of nsp.  Whole tiles come first, so the cut tiles are the last
+// (incomplete) round over the SMs: its few tiles are spread over all SMs instead of occupying a full tile time.
+struct Unit {
+  int t, sp, nsp, kb0, kb1;
+  __device__ __forceinline__ void set(const GemmParams& p, int u) {
+    if (u < p.full_tiles) { t = u; sp = 0; nsp = 1; }
+    else { const int r = u - p.full_tiles; t = p.full_tiles + r / p.k_splits; sp = r - (t - p.full_tiles) * p.k_splits; nsp = p.k_splits; }
+    kb0 = sp * p.num_k_blocks / nsp; kb1 = (sp + 1) * p.num_k_blocks / nsp;
+  }
 };
 
 template <int BN> struct GemmSmem {
@@ -130,7 +142,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (warp == 2) { ptx::tmem_alloc(tmem_slot, 2 * S::kAccStride); ptx::tmem_relinquish(); }
   grid_dependency_wait();
   grid_dependency_release();
-  int total_units = p.m_tiles * p.n_tiles * p.batch * p.k_splits;   // a unit = one tile, or one K slice of a tile
+  int total_units = p.full_tiles + (p.m_tiles * p.n_tiles * p.batch - p.full_tiles) * p.k_splits;   // a unit = one tile, or one K slice of a tile
   // A batch of requests of different sizes: the bounding grid (batch x largest request) is mostly holes, and
   // walking it leaves the SMs unevenly loaded.  Every CTA numbers the tiles that exist (a prefix over requests).
   __shared__ int tile_prefix[kMaxPrefixBatch + 1];
@@ -150,7 +162,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
-  if (use_prefix) total_units = tile_prefix[p.batch] * p.k_splits;
+  if (use_prefix) total_units = tile_prefix[p.batch] * p.k_splits;      // (the similarity cuts every tile or none)
   const uint32_t tmem_base = *tmem_slot;
   TileCoord<BN, EPI> tc;
   tc.prefix = use_prefix ? tile_prefix : nullptr;
@@ -167,12 +179,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       ptx::prefetch_tensormap(tm);
       int it = 0;                                   // k-blocks loaded so far, over all tiles
       bool ok = true;
+      Unit un;
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-        const int t = u / p.k_splits, sp = u - t * p.k_splits;
-        if (!tc.set(p, t)) continue;
+        un.set(p, u);
+        if (!tc.set(p, un.t)) continue;
         const int row0 = is_a ? tc.a_row : tc.b_row;
-        const int kb0 = sp * p.num_k_blocks / p.k_splits, kb1 = (sp + 1) * p.num_k_blocks / p.k_splits;
-        for (int kbk = kb0; kbk < kb1; ++kbk, ++it) {
+        for (int kbk = un.kb0; kbk < un.kb1; ++kbk, ++it) {
           const int s = it % kStages;
           ok = ptx::mbar_wait(&empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.dev_status);
           if (!ok) break;
@@ -194,10 +206,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const ptx::SmemDesc b_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(b_s));
       int it = 0, lt = 0;                           // k-blocks and tiles consumed so far
       bool ok = true;
+      Unit un;
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
-        const int t = u / p.k_splits, sp = u - t * p.k_splits;
-        if (!tc.set(p, t)) continue;
-        const int kb0 = sp * p.num_k_blocks / p.k_splits, kb1 = (sp + 1) * p.num_k_blocks / p.k_splits;
+        un.set(p, u);
+        if (!tc.set(p, un.t)) continue;
+        const int kb0 = un.kb0, kb1 = un.kb1;
         const int buf = lt & 1;
         ok = ptx::mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1, abort_flag, p.dev_status);   // epilogue done with it
         if (!ok) break;
@@ -227,8 +240,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int et = threadIdx.x - 64;               // 0..127 among the epilogue threads
     int lt = 0;
     __shared__ int s_prev;
+    Unit un;
     for (int u = blockIdx.x; u < total_units; u += gridDim.x) {
-      const int t = u / p.k_splits, sp = u - t * p.k_splits;
+      un.set(p, u);
+      const int t = un.t, sp = un.sp;
       if (!tc.set(p, t)) continue;
       const int buf = lt & 1;
       if (EPI == kEpiSim) {
@@ -241,13 +256,72 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!ok) break;
       ptx::tc_fence_after_sync();
       const uint32_t t_row = tmem_base + (uint32_t)buf * S::kAccStride + ((uint32_t)(quarter * 32) << 16);
-      if (EPI == kEpiProj) {
-        const int grow = tc.m0 + row;
+      // A tile whose K range is cut into slices on different SMs: every unit writes its partial sums out
+      // (column-major, so a warp's 32 rows are one 128-byte line); the unit that completes the tile (a
+      // counter, left at zero again) adds the parts in the order of the K slices and runs the epilogue on
+      // the sums: same values whichever unit comes last.
+      const bool split = un.nsp > 1;
+      const int ws_tile = t - p.full_tiles;                     // cut tiles are numbered from zero in the workspace
+      bool last = true;
+      if (split) {
+        float* part = p.split_ws + (size_t)(ws_tile * un.nsp + sp) * BN * kBM;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           uint32_t r[32];
           ptx::tmem_ld32(t_row + c, r);
           ptx::tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) part[(size_t)(c + i) * kBM + row] = __uint_as_float(r[i]);
+        }
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);          // the accumulator is free again
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0) s_prev = atomicAdd(p.split_counters + ws_tile, 1);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        last = s_prev == un.nsp - 1;
+        if (last) {
+          if (et == 0) p.split_counters[ws_tile] = 0;
+          __threadfence();
+        }
+      }
+      // 32 accumulator columns of this thread's row: from tensor memory, or the sum of the slices
+      auto load32 = [&](int c, float (&acc)[32]) {
+        if (!split) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_row + c, r);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = __uint_as_float(r[i]);
+        } else {
+          // all slices of the 32 columns are requested before any is added (one round trip, not one per slice)
+          float part[kMaxKSplits][32];
+#pragma unroll
+          for (int q = 0; q < kMaxKSplits; ++q) {
+            const float* src = p.split_ws + ((size_t)(ws_tile * un.nsp + q) * BN + c) * kBM + row;
+            if (q < un.nsp) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) part[q][i] = __ldcg(src + (size_t)i * kBM);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+#pragma unroll
+          for (int q = 0; q < kMaxKSplits; ++q)
+            if (q < un.nsp) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc[i] += part[q][i];
+            }
+        }
+      };
+      if (!last) { ++lt; continue; }
+      if (EPI == kEpiProj) {
+        const int grow = tc.m0 + row;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          float r[32];
+          load32(c, r);
           // 32 divides D, so a 32-column piece lies in one of q, k, v even when the tile straddles two of them
           const int gcol = tc.n0 + c, which = gcol / p.out_cols;
           __nv_bfloat16* dst = p.out[which] + (size_t)grow * p.out_cols + (gcol - which * p.out_cols) - c;
@@ -257,7 +331,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               uint32_t w[4];
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * j]), __uint_as_float(r[i + 2 * j + 1]));
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(r[i + 2 * j], r[i + 2 * j + 1]);
                 w[j] = *reinterpret_cast<uint32_t*>(&h2);
               }
               *reinterpret_cast<uint4*>(dst + c + i) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -268,9 +342,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int grow = tc.m0 + row;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
-          uint32_t r[32];
-          ptx::tmem_ld32(t_row + c, r);
-          ptx::tmem_wait_ld();
+          float r[32];
+          load32(c, r);
           if (grow < p.out_rows) {
             const size_t off = (size_t)grow * p.ld_out + tc.n0 + c;
 #pragma unroll
@@ -282,8 +355,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               }
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const float lo = __uint_as_float(r[i + 2 * j]) + __uint_as_float(w[j] << 16);
-                const float hi = __uint_as_float(r[i + 2 * j + 1]) + __uint_as_float(w[j] & 0xffff0000u);
+                const float lo = r[i + 2 * j] + __uint_as_float(w[j] << 16);
+                const float hi = r[i + 2 * j + 1] + __uint_as_float(w[j] & 0xffff0000u);
                 __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
                 w[j] = *reinterpret_cast<uint32_t*>(&h2);
               }
@@ -295,10 +368,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int grow = tc.m0 + row;
 #pragma unroll 1
         for (int c = 0; c < BN / 2; c += 32) {
-          uint32_t g[32], u[32];
-          ptx::tmem_ld32(t_row + c, g);
-          ptx::tmem_ld32(t_row + BN / 2 + c, u);
-          ptx::tmem_wait_ld();
+          float g[32], up[32];
+          load32(c, g);
+          load32(BN / 2 + c, up);
           if (grow < p.out_rows) {
             __nv_bfloat16* dst = p.lin_out + (size_t)grow * p.ld_out + tc.n0 + c;
 #pragma unroll
@@ -306,10 +378,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               uint32_t w[4];
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const float g0 = __uint_as_float(g[i + 2 * j]), g1 = __uint_as_float(g[i + 2 * j + 1]);
+                const float g0 = g[i + 2 * j], g1 = g[i + 2 * j + 1];
                 // silu(g) = g / (1 + exp(-g)); for very negative g the divisor is inf and the quotient 0
-                const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[i + 2 * j]);
-                const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[i + 2 * j + 1]);
+                const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * up[i + 2 * j];
+                const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * up[i + 2 * j + 1];
                 __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
                 w[j] = *reinterpret_cast<uint32_t*>(&h2);
               }
@@ -318,93 +390,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       } else {
-        // With few tiles each tile's K range is cut into k_splits units on different SMs.  Every unit
-        // writes its partial sums out (column-major, so a warp's 32 rows are one 128-byte line); the
-        // unit that completes the tile (a counter, left at zero again) adds the parts in the order of
-        // the K slices and runs the arg-max on the sums: same values whichever unit comes last.
-        const bool split = p.k_splits > 1;
-        bool last = true;
-        if (split) {
-          float* part = p.split_ws + (size_t)(t * p.k_splits + sp) * BN * kBM;
+        const int m = tc.m0 + row;
+        const int g = tc.v0 + m;
+        const bool active = m < tc.Vb && p.assign[g] < 0;     // a pruned token of this request
+        const float inm = active ? p.inv_norm[g] : 0.f;
+        float best_sim = -INFINITY;                        // strict > below: the lowest slot wins a tie
+        int best_slot = 0;
+        float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + tc.n0 : nullptr;
 #pragma unroll 1
-          for (int c = 0; c < BN; c += 32) {
-            uint32_t r[32];
-            ptx::tmem_ld32(t_row + c, r);
-            ptx::tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) part[(size_t)(c + i) * kBM + row] = __uint_as_float(r[i]);
-          }
-          ptx::tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);          // the accumulator is free again
-          __threadfence();
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (et == 0) s_prev = atomicAdd(p.split_counters + t, 1);
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          last = s_prev == p.k_splits - 1;
-          if (last) {
-            if (et == 0) p.split_counters[t] = 0;
-            __threadfence();
-          }
-        }
-        if (last) {
-          const int m = tc.m0 + row;
-          const int g = tc.v0 + m;
-          const bool active = m < tc.Vb && p.assign[g] < 0;     // a pruned token of this request
-          const float inm = active ? p.inv_norm[g] : 0.f;
-          float best_sim = -INFINITY;                        // strict > below: the lowest slot wins a tie
-          int best_slot = 0;
-          float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + tc.n0 : nullptr;
-#pragma unroll 1
-          for (int c = 0; c < BN; c += 32) {
-            float dot[32];
-            if (!split) {
-              uint32_t r[32];
-              ptx::tmem_ld32(t_row + c, r);
-              ptx::tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) dot[i] = __uint_as_float(r[i]);
-            } else {
-              // all slices of the 32 columns are requested before any is added (one round trip, not k_splits)
-              float part[kMaxKSplits][32];
-#pragma unroll
-              for (int q = 0; q < kMaxKSplits; ++q) {
-                const float* src = p.split_ws + ((size_t)(t * p.k_splits + q) * BN + c) * kBM + row;
-                if (q < p.k_splits) {
-#pragma unroll
-                  for (int i = 0; i < 32; ++i) part[q][i] = __ldcg(src + (size_t)i * kBM);
-                }
-              }
-#pragma unroll
-              for (int i = 0; i < 32; ++i) dot[i] = 0.f;
-#pragma unroll
-              for (int q = 0; q < kMaxKSplits; ++q)
-                if (q < p.k_splits) {
-#pragma unroll
-                  for (int i = 0; i < 32; ++i) dot[i] += part[q][i];
-                }
-            }
-            if (active) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const int sidx = tc.n0 + c + i;
-                if (sidx < tc.kb) {
-                  // the value the arg-max compares; + 0 turns a negative zero into the positive one
-                  const float sim = (dot[i] * inm) * ink_s[c + i] + 0.0f;
-                  if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
-                  if (dbg != nullptr) dbg[c + i] = sim;
-                }
-              }
-            }
-          }
+        for (int c = 0; c < BN; c += 32) {
+          float dot[32];
+          load32(c, dot);
           if (active) {
-            const unsigned long long mine =
-                ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
-            atomicMax(p.best + g, mine);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int sidx = tc.n0 + c + i;
+              if (sidx < tc.kb) {
+                // the value the arg-max compares; + 0 turns a negative zero into the positive one
+                const float sim = (dot[i] * inm) * ink_s[c + i] + 0.0f;
+                if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
+                if (dbg != nullptr) dbg[c + i] = sim;
+              }
+            }
           }
         }
-        if (split) { ++lt; continue; }
+        if (active) {
+          const unsigned long long mine =
+              ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
+          atomicMax(p.best + g, mine);
+        }
       }
+      if (split) { ++lt; continue; }                      // (its accumulator was released when the partial went out)
       // the accumulator may be overwritten once all four warps have read it
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -433,11 +449,36 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
+// The dense layers walk whole tiles; when the last round over the SMs is incomplete, its tiles are cut into K
+// slices so that the round costs a fraction of a tile time plus the exchange of partial sums.  Costs in units of
+// one k-block of main loop (about 0.35 us): the exchange costs about 30 + 5 per slice (measured: 15 - 18 us, most of
+// it the 128 threads of the completing unit reading the other slices back, 64 KB in flight per round trip), so it
+// pays for long K only: the down projection of the feed-forward network, not the 64-k-block projections.
+void plan_tail_split(const d3tom_ctx* ctx, GemmParams& p) {
+  const int tiles = p.m_tiles * p.n_tiles * p.batch, sms = ctx->sm_count;
+  p.k_splits = 1; p.full_tiles = tiles;
+  const int rem = tiles % sms;
+  if (rem == 0 || p.split_ws == nullptr) return;
+  int best = p.num_k_blocks, best_s = 1;
+  for (int sp = 2; sp <= kMaxKSplits; ++sp) {
+    if (p.num_k_blocks / sp < 8 || rem * sp > 2 * sms) break;      // slices too short / more parts than the workspace holds
+    const int rounds = (rem * sp + sms - 1) / sms;
+    const int cost = rounds * ((p.num_k_blocks + sp - 1) / sp) + 30 + 5 * sp;
+    if (cost < best) { best = cost; best_s = sp; }
+  }
+  if (best_s > 1) { p.k_splits = best_s; p.full_tiles = tiles - rem; }
+}
+
 template <int BN, int EPI>
-int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, const GemmParams& p, cudaStream_t s) {
-  const long long tiles = (long long)p.m_tiles * p.n_tiles * p.batch * p.k_splits;
-  if (tiles <= 0) return D3TOM_OK;
-  const int grid = (int)(tiles < ctx->sm_count ? tiles : ctx->sm_count);          // persistent: one CTA per SM
+int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t s) {
+  if (EPI != kEpiSim) {
+    p.split_ws = ctx->gemm_split_ws; p.split_counters = ctx->gemm_split_counters;
+    plan_tail_split(ctx, p);
+  }
+  const long long tiles = (long long)p.m_tiles * p.n_tiles * p.batch;
+  const long long units = p.full_tiles + (tiles - p.full_tiles) * p.k_splits;
+  if (units <= 0) return D3TOM_OK;
+  const int grid = (int)(units < ctx->sm_count ? units : ctx->sm_count);          // persistent: one CTA per SM
   D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            GemmSmem<BN>::kBytes));
   D3TOM_CUDA_TRY(ctx, launch_serialized(gemm_tc_kernel<BN, EPI>, grid, kGemmThreads, GemmSmem<BN>::kBytes, s, ta, tb, p));
@@ -559,6 +600,7 @@ int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
     if (splits > p.num_k_blocks) splits = p.num_k_blocks;
     if (splits < 2 || tiles * splits > 2LL * ctx->sm_count) splits = 1;
     p.k_splits = splits;
+    p.full_tiles = 0;                                   // every tile is cut (or none: one slice)
     p.split_ws = ctx->gemm_split_ws; p.split_counters = ctx->gemm_split_counters;
   }
   if (a.max_kept > 128) {      // 256-wide tiles: the A tile is streamed once per 256 kept rows and each MMA covers twice the work

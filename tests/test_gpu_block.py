@@ -49,6 +49,13 @@ def test_linear_bf16_without_residual_and_in_place():
     run_linear(1, 64, 128, "bf16", residual=True)
 
 
+def test_linear_and_ffn_bf16_long_k_few_tiles_cut_into_k_slices():
+    # six tiles for 148 SMs and 64 k-blocks: the tiles of the (only, incomplete) round are cut into K slices whose
+    # partial sums meet in the workspace; the same for the gate/up pass of the feed-forward network
+    run_linear(300, 4096, 512, "bf16", residual=True, seed=3)
+    run_ffn(300, 4096, 256, "bf16", seed=4)
+
+
 def test_linear_fp32_odd_sizes():
     run_linear(70, 50, 45, "fp32", residual=True)
     run_linear(33, 7, 3, "fp32", residual=False)
