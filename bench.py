@@ -40,7 +40,7 @@ WORKLOAD_TEXT = {
 }
 # DRAM bytes of one launch of the dominant kernel from the committed ncu capture (null for configs not captured,
 # and to be reset to null whenever attn_tc.cu changes after the capture)
-ATTN_TRAFFIC_BYTES = {"C2": 161.1e6}
+ATTN_TRAFFIC_BYTES = {"C2": 164.8e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
