@@ -267,7 +267,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-block", action="store_true", help="skip the timing of the rest of a post-merge block")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
-    ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "step"],
+    ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
                     help="profiling aid: after one full step, run just this call --steps times and exit")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -402,6 +402,16 @@ def main():
                                                               step.layer_out[0]),
             "step": run,
         }
+        if args.only in ("proj_out", "ffn"):          # the rest of a post-merge block at the shortened length
+            m_ff = 3 * step.D
+            t = wl.block_inputs(1000, 8, step.D, m_ff, w.dtype)
+            w_o, w_gu, w_dn = t["w_o"].to(dev), t["w_gate_up"].to(dev), t["w_down"].to(dev)
+            act = torch.empty(step.total_out, m_ff, dtype=q.dtype, device=dev)
+            y = torch.empty(step.total_out, step.D, dtype=q.dtype, device=dev)
+            calls["proj_out"] = lambda: step.ctx.d3tom_linear(step.layer_out[0], w_o, step.hidden_out, step.total_out,
+                                                              step.D, step.D, y)
+            calls["ffn"] = lambda: step.ctx.d3tom_ffn(step.hidden_out, w_gu, w_dn, step.hidden_out, step.total_out,
+                                                      step.D, m_ff, act, y)
         torch.cuda.synchronize()
         us = timed(calls[args.only], args.steps)
         print(json.dumps({"only": args.only, "us": us, "config": args.config}))
