@@ -266,6 +266,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-block", action="store_true", help="skip the timing of the rest of a post-merge block")
+    ap.add_argument("--tokens-per-step", type=int, default=1,
+                    help="schedule config: response tokens revealed per denoising step (2 gives T = 32 for 64 tokens)")
+    ap.add_argument("--reversed", action="store_true", help="schedule config: the high->low ablation of the schedule")
+    ap.add_argument("--deciders", default="all", choices=["all", "recent"],
+                    help="schedule config: every token revealed so far, or only those of the previous step")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
     ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
                     help="profiling aid: after one full step, run just this call --steps times and exit")
@@ -312,6 +317,7 @@ def main():
     from paper_2511_12280_b200 import binding as B_
     from paper_2511_12280_b200.pipeline import MergeLayerStep
     from paper_2511_12280_b200 import replicas
+    from paper_2511_12280_b200 import trajectory
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the merge-layer path has no CPU fallback")
@@ -325,15 +331,19 @@ def main():
     config["requests_per_gpu"] = w.B
     total = int(w.cu_seqlens[-1])
     # one problem per schedule step (a single one for the constant-ratio configs)
+    plan = plan_unmerged = None
     if w.T:
         a_min, a_max = 2.0 * (1.0 - w.mean_keep_ratio) - 1.0, 1.0
-        dec_steps = [w.step_deciders(s) for s in range(w.T)]
-        keep_steps = []
-        for s, dec in enumerate(dec_steps):
-            alpha = B_.d3tom_schedule_alpha(s, w.T, a_min, a_max)
-            # a step without deciders runs unmerged (Algorithm 1, else-branch)
-            keep_steps.append([B_.d3tom_keep_count(w.n_visual[0], 1.0 - alpha) if len(dec[0]) else w.n_visual[0]])
-        config["schedule"] = {"T": w.T, "alpha_min": a_min, "alpha_max": a_max, "keep_counts": [k[0] for k in keep_steps]}
+        T_steps = w.T // args.tokens_per_step
+        kw_plan = dict(tokens_per_step=args.tokens_per_step, reversed_=args.reversed, deciders=args.deciders)
+        plan = trajectory.plan_schedule(w.n_visual, w.n_prompt, [w.decode_order], T_steps, a_min, a_max, **kw_plan)
+        plan_unmerged = trajectory.plan_schedule(w.n_visual, w.n_prompt, [w.decode_order], T_steps, a_min, a_max,
+                                                 merged=False, **kw_plan)
+        dec_steps = [p.decider_pos for p in plan]
+        keep_steps = [p.keep_count for p in plan]
+        config["schedule"] = {"T": T_steps, "alpha_min": a_min, "alpha_max": a_max, "tokens_per_step": args.tokens_per_step,
+                              "reversed": bool(args.reversed), "deciders": args.deciders,
+                              "keep_counts": [k[0] for k in keep_steps]}
     else:
         dec_steps = [w.decider_pos]
         keep_steps = [[B_.d3tom_keep_count(v, r) for v, r in zip(w.n_visual, w.keep_ratio)]]
@@ -436,6 +446,17 @@ def main():
                 counter["i"] = 0
                 series.append([timed(run, 1) for _ in range(n_prob)])
             per_step = [float(x) for x in np.median(np.asarray(series), axis=0)]
+            # the same trajectory without merging (every visual token kept), one graph per step as well
+            traj_u = trajectory.Trajectory(step, plan_unmerged, w.n_visual, w.n_prompt, w.n_resp)
+            traj_m = trajectory.Trajectory(step, plan, w.n_visual, w.n_prompt, w.n_resp)
+            traj_u.capture(qs, k, v, w_post)
+            traj_u.run()
+            sync_all()
+            unmerged_us = float(np.median([timed(traj_u.run, 1) for _ in range(3)]))
+            traj_info = {"T": len(plan), "total_us": float(sum(per_step)), "unmerged_total_us": unmerged_us,
+                         "time_ratio": float(sum(per_step)) / unmerged_us,
+                         "flops_ratio": traj_m.flops(step.D, step.n_post) / traj_u.flops(step.D, step.n_post)}
+            del traj_u
         # the breakdown below is taken at the middle problem
         counter["i"] = n_prob // 2
         run()
@@ -547,6 +568,7 @@ def main():
     if per_step is not None:
         line["per_step_us"] = per_step
         line["trajectory_total_us"] = float(sum(per_step))
+        line["trajectory"] = traj_info
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         kw = {}
         if w.T:
