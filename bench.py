@@ -464,6 +464,12 @@ def main():
         # ---- per-call breakdown (each call timed back to back on warm instruction caches;
         #      every call's working set is streamed from HBM or L2 as it would be inside the step)
         reps = min(100, max(10, args.steps))
+        # the dominant kernel alone (no importance side-work): the attention kernel at the merge-layer length; taken
+        # first, before the long GEMM timings below pull the board into its power cap
+        sync_all()
+        time.sleep(0.5)      # the burst peak it is compared with was measured on an idle board: let the power state settle
+        attn_kernel_us = timed(lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
+                                                                  step.max_seqlen, step.scale, step.attn_out), reps)
         br = {}
         br["attn_importance"] = timed(lambda: step.attn_importance(q, k, v), reps)
         br["select"] = timed(lambda: step.select(), reps)
@@ -483,9 +489,6 @@ def main():
             block = block_timings(step, w, w_post[0], q, k, v, dev, timed, max(5, reps // 4))
             br["proj_out"] = block["Nm"]["proj_out"]
             br["ffn"] = block["Nm"]["ffn"]
-        # the dominant kernel alone (no importance side-work): the attention kernel at the merge-layer length
-        attn_kernel_us = timed(lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
-                                                                  step.max_seqlen, step.scale, step.attn_out), reps)
         sync_all()
     clocks = clk.summary()
     assert step.ctx.device_status() == 0, "device status word reports a kernel-side problem"
