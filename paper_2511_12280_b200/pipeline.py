@@ -147,3 +147,68 @@ class MergeLayerStep:
         aggregate/compact), and 2 per post-merge layer."""
         sim = 1 if self.total_out < self.total else 0
         return 2 + 1 + 1 + sim + 2 + 2 * self.n_post
+
+
+class HostFedStep:
+    """Runs merge-layer steps whose Q, K, V live in pinned host memory and whose result goes back to the host.
+
+    Three streams: the inputs of step i + 1 are copied to the device (two input slots) while step i computes on
+    the caller's current stream, and the result of step i leaves on a third stream while step i + 1 computes, so
+    a sequence of steps costs max(copy, compute) per step instead of their sum.  ``submit`` only enqueues;
+    ``wait`` makes the caller's current stream wait for the last result copy.  With ``use_graphs`` every
+    (problem, slot) pair is recorded once as a CUDA graph and replayed."""
+
+    def __init__(self, step: MergeLayerStep, like: torch.Tensor, w_post: Optional[Sequence[torch.Tensor]] = None,
+                 use_graphs: bool = True):
+        self.step, self.w_post, self.use_graphs = step, w_post, use_graphs
+        dev = step.dev
+        self.slots = [SimpleNamespace(q=torch.empty(like.shape, dtype=like.dtype, device=dev),
+                                      k=torch.empty(like.shape, dtype=like.dtype, device=dev),
+                                      v=torch.empty(like.shape, dtype=like.dtype, device=dev)) for _ in range(2)]
+        self.copy_stream = torch.cuda.Stream(device=dev)
+        self.out_stream = torch.cuda.Stream(device=dev)
+        self.copied = [torch.cuda.Event() for _ in range(2)]
+        self.consumed = [torch.cuda.Event() for _ in range(2)]
+        self.computed, self.out_done = torch.cuda.Event(), torch.cuda.Event()
+        self.graphs = {}
+        self.n = 0
+
+    def submit(self, q_h, k_h, v_h, out_h, problem, key=None):
+        """q_h, k_h, v_h: pinned host tensors shaped like the slots; out_h: pinned host tensor that receives the
+        rows of the last tensor of the chain; problem: from ``MergeLayerStep.make_problem``; key: a hashable
+        name of the problem for the graph cache (defaults to its identity)."""
+        step = self.step
+        s = self.n & 1
+        self.n += 1
+        slot = self.slots[s]
+        cur = torch.cuda.current_stream(step.dev)
+        with torch.cuda.stream(self.copy_stream):
+            self.copy_stream.wait_event(self.consumed[s])       # the step that last read this slot has run
+            slot.q.copy_(q_h, non_blocking=True)
+            slot.k.copy_(k_h, non_blocking=True)
+            slot.v.copy_(v_h, non_blocking=True)
+            self.copied[s].record(self.copy_stream)
+        step.use_problem(problem)
+        gkey = (id(problem) if key is None else key, s)
+        if self.use_graphs and gkey not in self.graphs:
+            # recorded once per (problem, slot); recording runs the step, so everything in flight finishes first
+            torch.cuda.synchronize(step.dev)
+            self.graphs[gkey] = step.capture(slot.q, slot.k, slot.v, self.w_post)
+        cur.wait_event(self.copied[s])
+        cur.wait_event(self.out_done)                           # the previous result has left the output buffers
+        if self.use_graphs:
+            self.graphs[gkey].replay()
+            y = step.layer_out[-1] if step.n_post else step.hidden_out
+        else:
+            y = step.run(slot.q, slot.k, slot.v, self.w_post)
+        self.consumed[s].record(cur)
+        self.computed.record(cur)
+        n = step.total_out
+        with torch.cuda.stream(self.out_stream):
+            self.out_stream.wait_event(self.computed)
+            out_h[:n].copy_(y[:n], non_blocking=True)
+            self.out_done.record(self.out_stream)
+        return n
+
+    def wait(self):
+        torch.cuda.current_stream(self.step.dev).wait_event(self.out_done)
