@@ -115,6 +115,21 @@ class MergeLayerStep:
         self.ctx.d3tom_attn_varlen(self.q2, self.k2, self.v2, self.cu_out, self.nB, self.total_out, self.max_out,
                                    self.scale, self.layer_out[l], stream)
 
+    def post_block(self, l: int, x, w_qkv, w_o, w_gate_up, w_down, stream=None):
+        """A whole post-merge block on the shortened sequence (Algorithm 1, the layers after l*; layer-cost
+        equation): attention as in post_layer, then x1 = x + attn W_o^T and y = x1 + FFN(x1), written to
+        layer_out[l].  The activation scratch [rows, m] is allocated on first use."""
+        m = w_down.shape[1]
+        if getattr(self, "ffn_act", None) is None or self.ffn_act.shape[1] != m:
+            self.ffn_act = torch.empty(self.attn_out.shape[0], m, dtype=self.dtype, device=self.dev)
+            self.block_x1 = torch.empty_like(self.attn_out)
+        self.post_layer(l, x, w_qkv, stream)
+        n = self.total_out
+        self.ctx.d3tom_linear(self.layer_out[l], w_o, x, n, self.D, self.D, self.block_x1, stream)
+        self.ctx.d3tom_ffn(self.block_x1, w_gate_up, w_down, self.block_x1, n, self.D, m, self.ffn_act,
+                           self.layer_out[l], stream)
+        return self.layer_out[l]
+
     def run(self, q, k, v, w_post: Optional[Sequence[torch.Tensor]] = None, stream=None):
         """Enqueue the whole step.  Returns the last tensor of the chain."""
         self.attn_importance(q, k, v, stream)

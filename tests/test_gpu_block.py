@@ -134,3 +134,30 @@ def test_unsupported_shapes_and_bad_arguments_are_refused_on_the_host():
     torch.cuda.synchronize()
     assert ctx.device_status() == 0
     ctx.close()
+
+
+def test_whole_post_merge_block_after_a_merge_step():
+    # merge-layer step, then one LLaDA-shaped block (attention, output projection, gated FFN, two residuals) on the
+    # shortened ragged batch; every stage is checked against the oracle fed with the GPU's previous stage
+    w = wl.make_workload("blk", "bf16", 2, 128, 41, 16, [dict(V=300, P=17, O=24, n_dec=5, r=0.3),
+                                                          dict(V=200, P=9, O=8, n_dec=2, r=0.5)], post_layers=1)
+    step = pu.make_step(w, sim_debug=False)
+    dev = step.dev
+    D, m = step.D, 384
+    t = wl.block_inputs(7, 8, D, m, "bf16")
+    w_o, w_gu, w_dn = t["w_o"] * 2, t["w_gate_up"] * 4, t["w_down"] * 4
+    q, k, v = w.q_for().to(dev), w.k.to(dev), w.v.to(dev)
+    step.attn_importance(q, k, v); step.select(); step.merge()
+    x = step.hidden_out
+    y = step.post_block(0, x, w.w_post[0].to(dev), w_o.to(dev), w_gu.to(dev), w_dn.to(dev))
+    torch.cuda.synchronize()
+    assert step.ctx.device_status() == 0
+    n = step.total_out
+    xg = pu.f64(x)[:n]
+    attn = orc.post_layer(xg, pu.f64(w.w_post[0]), step.cu_out_h, w.H, "bf16").reshape(n, D)
+    x1 = orc.linear(attn, pu.f64(w_o), xg, "bf16")
+    pu.assert_close(pu.f64(step.block_x1)[:n], x1, "bf16", "x + attn W_o")
+    x1g = pu.f64(step.block_x1)[:n]
+    want, _ = orc.ffn(x1g, pu.f64(w_gu), pu.f64(w_dn), x1g, "bf16")
+    pu.assert_close(pu.f64(y)[:n], want, "bf16", "block output")
+    step.ctx.close()
