@@ -497,12 +497,9 @@ int launch_sim_simt(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
 }
 
 int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(members_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kMemberSmemSlots * (int)sizeof(int) + kBitmapBytes));
-    attr_set = true;
-  }
+  // (the attribute belongs to the current device: set on every call, a process may drive several GPUs)
+  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(members_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           kMemberSmemSlots * (int)sizeof(int) + kBitmapBytes));
   // shared memory of the members kernel: counters when they fit, then one position bitmap per sorting warp
   const int ctr_ints = a.max_kept <= kMemberSmemSlots ? a.max_kept : 0;
   const int words = ceil_div(a.max_visual > 0 ? a.max_visual : 1, 32);

@@ -150,11 +150,8 @@ int launch_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis
                   cudaStream_t s) {
   const size_t smem = (size_t)max_visual * sizeof(uint32_t);
   if (smem <= 160 * 1024) {
-    static bool attr_set = false;
-    if (!attr_set) {
-      D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-      attr_set = true;
-    }
+    // (the attribute belongs to the current device: set on every call, a process may drive several GPUs)
+    D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
     D3TOM_CUDA_TRY(ctx, launch_serialized(select_kernel<true>, B, kThreads, smem, s, importance, cu_vis, keep_count, cu_kept, kept_idx, keep_mask));
   } else {
     D3TOM_CUDA_TRY(ctx, launch_serialized(select_kernel<false>, B, kThreads, 0, s, importance, cu_vis, keep_count, cu_kept, kept_idx, keep_mask));
