@@ -193,12 +193,37 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
   unsigned* bitmaps = reinterpret_cast<unsigned*>(dyn_s + ctr_ints);
   __shared__ int warp_tot[32];
   __shared__ int carry;
+  // the request's heavy kept tokens, so that the sorting warps below need not walk over all kept tokens
+  constexpr int kHeavyLocal = 2048;
+  __shared__ int heavy_local[kHeavyLocal];
+  __shared__ int n_heavy_local;
+  if (tid == 0) n_heavy_local = 0;
   for (int s = tid; s < kb; s += kMemberThreads) ctr[s] = 0;
   __syncthreads();
-  for (int m = tid; m < V; m += kMemberThreads) {
+  // requests of up to kSlotRegs x 1024 visual tokens keep every token's slot in a register between the counting
+  // pass and the filling pass (one round trip to global memory less); -1: a kept token
+  constexpr int kSlotRegs = 8;
+  const bool in_regs = V <= kSlotRegs * kMemberThreads;
+  int my_slot[kSlotRegs];
+#pragma unroll
+  for (int i = 0; i < kSlotRegs; ++i) {
+    my_slot[i] = -1;
+    const int m = tid + i * kMemberThreads;
+    if (in_regs && m < V) {
+      const unsigned long long w = best[v0 + m];
+      if (w != 0ull) my_slot[i] = (int)(0xffffffffu - (unsigned)(w & 0xffffffffull));   // a pruned token (kept tokens keep best == 0)
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kSlotRegs; ++i)
+    if (my_slot[i] >= 0) {
+      assign[v0 + tid + i * kMemberThreads] = my_slot[i];
+      atomicAdd(&ctr[my_slot[i]], 1);
+    }
+  for (int m = tid; m < V && !in_regs; m += kMemberThreads) {
     const int g = v0 + m;
     const unsigned long long w = best[g];
-    if (w != 0ull) {                               // a pruned token (kept tokens keep best == 0)
+    if (w != 0ull) {
       const int slot = (int)(0xffffffffu - (unsigned)(w & 0xffffffffull));
       assign[g] = slot;
       atomicAdd(&ctr[slot], 1);
@@ -235,7 +260,11 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
       member_count[k0 + s] = c;
       member_off[k0 + s] = pruned_base + excl;
       ctr[s] = pruned_base + excl;
-      if (c >= kHeavy) heavy_slots[atomicAdd(n_heavy, 1)] = k0 + s;
+      if (c >= kHeavy) {
+        heavy_slots[atomicAdd(n_heavy, 1)] = k0 + s;
+        const int li = atomicAdd(&n_heavy_local, 1);
+        if (li < kHeavyLocal) heavy_local[li] = s;
+      }
       // what the aggregation needs to know about this output row, in one 16-byte record
       row_desc[out0 + s] = make_int4(lo + kept_idx[k0 + s], c, pruned_base + excl, lo);
     }
@@ -243,7 +272,10 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
     if (tid == 0) carry += chunk_total;
     __syncthreads();
   }
-  for (int m = tid; m < V; m += kMemberThreads) {
+#pragma unroll
+  for (int i = 0; i < kSlotRegs; ++i)
+    if (my_slot[i] >= 0) member_list[atomicAdd(&ctr[my_slot[i]], 1)] = tid + i * kMemberThreads;
+  for (int m = tid; m < V && !in_regs; m += kMemberThreads) {
     const int g = v0 + m;
     if (best[g] != 0ull) member_list[atomicAdd(&ctr[assign[g]], 1)] = m;
   }
@@ -252,7 +284,10 @@ members_kernel(const int32_t* __restrict__ cu_vis, const int32_t* __restrict__ c
   if (warp < bitmap_warps) {
     const int words = (V + 31) >> 5;
     unsigned* bm = bitmaps + (size_t)warp * words;
-    for (int s = warp; s < kb; s += bitmap_warps) {
+    const int nh = n_heavy_local;
+    const bool listed = nh <= kHeavyLocal;         // else (more heavy tokens than the list holds): walk over all kept tokens
+    for (int h = warp; h < (listed ? nh : kb); h += bitmap_warps) {
+      const int s = listed ? heavy_local[h] : h;
       const int cnt = member_count[k0 + s];
       if (cnt < kHeavy) continue;                  // uniform over the warp
       const int off = member_off[k0 + s];
