@@ -123,7 +123,8 @@ importance_finish_kernel(const float* __restrict__ score, const float2* __restri
     }
     __syncthreads();
     const float* col = score + ((size_t)h * max_deciders + dc) * vis_stride + jj;
-#pragma unroll 8
+    // (the loads of 16 deciders are in flight together; the sum still runs in ascending decider order)
+#pragma unroll 16
     for (int d = 0; d < nd; ++d)
       acc = fmaf(exp2f(fmaf(col[(size_t)d * vis_stride], scale_log2, neg_m[d])), inv_l[d], acc);
   }
@@ -141,6 +142,7 @@ importance_finish_kernel(const float* __restrict__ score, const float2* __restri
   if (is_last && j < Vb) {
     __threadfence();
     float tot = 0.f;
+#pragma unroll 8
     for (int hh = 0; hh < H; ++hh) tot += __ldcg(partial + (size_t)hh * partial_stride + g0 + j);
     importance[g0 + j] = tot;
   }
