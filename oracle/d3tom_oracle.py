@@ -138,7 +138,10 @@ def importance(q, k, cu_seqlens, n_visual, decider_pos, cu_deciders, scale):
 def keep_count(n_visual: int, keep_ratio: float) -> int:
     """Number of tokens with Rank <= (1 - alpha)|V|: floor(r*|V| + 1e-9),
     clamped to [1, |V|].  The 1e-9 guards products such as (1-0.9)*1000 that
-    land just below an integer in binary."""
+    land just below an integer in binary.  A request without visual tokens
+    (|V| = 0, where the clamp has no meaning) keeps nothing."""
+    if n_visual <= 0:
+        return 0
     k = int(np.floor(keep_ratio * n_visual + 1e-9))
     return max(1, min(int(n_visual), k))
 

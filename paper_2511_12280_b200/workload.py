@@ -138,7 +138,10 @@ def make_workload(name, dtype, H, dh, seed, n_clusters, requests, post_layers=0,
             dec = np.zeros(0, dtype=np.int32)
         else:
             dec = np.sort(rng.choice(O, size=n_dec, replace=False)).astype(np.int32) + (V + P)
-        sal = np.sort(rng.choice(V, size=max(1, int(round(SALIENT_FRACTION * V))), replace=False)).astype(np.int32)
+        if V > 0:
+            sal = np.sort(rng.choice(V, size=max(1, int(round(SALIENT_FRACTION * V))), replace=False)).astype(np.int32)
+        else:
+            sal = np.zeros(0, dtype=np.int32)       # a text-only request: nothing to merge
         u = _normal(rng, (H, dh))
         u /= np.linalg.norm(u, axis=1, keepdims=True)
         u = torch.from_numpy(u)

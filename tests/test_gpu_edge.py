@@ -64,6 +64,14 @@ def test_kept_set_larger_than_the_shared_memory_counters():
     pu.check_step(w, full_attention=False, n_sample_rows=6)
 
 
+def test_text_only_request_inside_a_batch():
+    # a request without visual tokens between two ordinary ones: nothing to select or merge there, its rows are
+    # copied, its attention runs as usual
+    w = small(reqs=[dict(V=140, P=9, O=8, n_dec=2, r=0.5), dict(V=0, P=20, O=8, n_dec=2, r=0.5),
+                    dict(V=130, P=5, O=8, n_dec=3, r=0.25)])
+    pu.check_step(w)
+
+
 def test_keep_ratio_one_is_identity():
     w = small(post=0)
     step = pu.make_step(w, keep_count=list(w.n_visual), sim_debug=False)

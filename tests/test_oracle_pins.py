@@ -485,3 +485,9 @@ def test_ffn_activation_is_rounded_to_storage_before_the_second_product():
     assert np.array_equal(y, act)
     exact = orc.silu(x @ wgu[:m].T) * (x @ wgu[m:].T)
     assert np.array_equal(act, orc.round_bf16(exact)) and not np.array_equal(act, exact)
+
+
+def test_keep_count_of_a_request_without_visual_tokens_is_zero():
+    assert orc.keep_count(0, 0.5) == 0 and orc.keep_count(0, 1.0) == 0
+    assert orc.keep_count(1, 0.01) == 1          # the clamp to one token needs a token
+    assert len(orc.select(np.zeros(0), 0)) == 0
