@@ -451,8 +451,9 @@ EncodeTiledFn get_encode_fn() {
 
 // The dense layers walk whole tiles; when the last round over the SMs is incomplete, its tiles are cut into K
 // slices so that the round costs a fraction of a tile time plus the exchange of partial sums.  Costs in units of
-// one k-block of main loop (about 0.35 us): the exchange costs about 30 + 5 per slice (measured: 15 - 18 us, most of
-// it the 128 threads of the completing unit reading the other slices back, 64 KB in flight per round trip), so it
+// one k-block of main loop (about 0.35 us): a cut round costs about 30 + 5 per slice on top of its k-blocks (measured:
+// 15 - 18 us; reading the slices back through bulk copies instead of register loads did not change it, so it is the
+// cold start of the short main loops and the fence / counter round trips rather than the read-back), so cutting
 // pays for long K only: the down projection of the feed-forward network, not the 64-k-block projections.
 void plan_tail_split(const d3tom_ctx* ctx, GemmParams& p) {
   const int tiles = p.m_tiles * p.n_tiles * p.batch, sms = ctx->sm_count;
