@@ -65,16 +65,21 @@ struct Unit {
   }
 };
 
-template <int BN> struct GemmSmem {
-  static constexpr int kStages = BN == 256 ? 4 : (BN == 192 ? 5 : 6);   // as many as fit in 227 KB
+// MT = 1: a CTA tile is 128 x BN with two accumulators (the epilogue of a tile overlaps the main loop of the next).
+// MT = 2: a CTA tile is 256 x BN: two 128-row A tiles share every B tile in shared memory, so a k-block moves
+//         32 + 32 KB for 1024 tensor cycles (62 B/clk) where the 128 x 256 tile moves 16 + 32 KB for 512 (96 B/clk);
+//         the dense layers are bound by what the SMs can pull out of L2, so this is the faster shape whenever there
+//         are enough rows.  Both accumulators belong to the one tile (no overlap of epilogue and main loop).
+template <int BN, int MT = 1> struct GemmSmem {
+  static constexpr int kABytes = MT * kBM * kBK * 2, kBBytes = BN * kBK * 2;
+  static constexpr int kStages = (MT == 2) ? 3 : (BN == 256 ? 4 : (BN == 192 ? 5 : 6));   // as many as fit in 227 KB
   static constexpr int kAccStride = BN <= 128 ? 128 : 256;              // TMEM columns between the two accumulators
-  static constexpr int kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2;
   static constexpr int kBytes = kStages * (kABytes + kBBytes) + 1024 /*alignment slack*/ + 256 /*barriers*/ + BN * 4;
 };
 
 // Where tile `t` of the walk lies: rows of A, rows of B, and for the similarity the request
 // it belongs to.  Returns false for a tile of the bounding grid that a request does not reach.
-template <int BN, int EPI>
+template <int BN, int EPI, int MT = 1>
 struct TileCoord {
   int m0, n0, a_row, b_row, b, Vb, kb, v0, k0;
   const int* prefix;      // similarity with a ragged batch: tiles before request b (shared memory), or null
@@ -99,7 +104,7 @@ struct TileCoord {
     ni = rest % p.n_tiles;
     b = rest / p.n_tiles;
     // (a gate-up tile covers BN / 2 output features: its B rows are 128 gate rows and 128 up rows)
-    m0 = mi * kBM; n0 = ni * (EPI == kEpiGateUp ? BN / 2 : BN); a_row = m0; b_row = n0;
+    m0 = mi * (MT * kBM); n0 = ni * (EPI == kEpiGateUp ? BN / 2 : BN); a_row = m0; b_row = n0;
     Vb = kb = v0 = k0 = 0;
     if (EPI == kEpiSim) {
       v0 = p.cu_vis[b]; Vb = p.cu_vis[b + 1] - v0;
@@ -114,10 +119,11 @@ struct TileCoord {
 
 constexpr int kMaxPrefixBatch = 64;     // ragged batches up to this many requests number only the tiles that exist
 
-template <int BN, int EPI>
+template <int BN, int EPI, int MT = 1>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
-  using S = GemmSmem<BN>;
+  static_assert(MT == 1 || (BN == 256 && EPI != kEpiSim), "the 256-row tile serves the dense layers at 256 columns");
+  using S = GemmSmem<BN, MT>;
   constexpr int kStages = S::kStages;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -164,7 +170,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   ptx::tc_fence_after_sync();
   if (use_prefix) total_units = tile_prefix[p.batch] * p.k_splits;      // (the similarity cuts every tile or none)
   const uint32_t tmem_base = *tmem_slot;
-  TileCoord<BN, EPI> tc;
+  TileCoord<BN, EPI, MT> tc;
   tc.prefix = use_prefix ? tile_prefix : nullptr;
 
   if (warp == 0 || warp == 6) {
@@ -211,8 +217,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         un.set(p, u);
         if (!tc.set(p, un.t)) continue;
         const int kb0 = un.kb0, kb1 = un.kb1;
-        const int buf = lt & 1;
-        ok = ptx::mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1, abort_flag, p.dev_status);   // epilogue done with it
+        const int buf = MT == 2 ? 0 : (lt & 1);               // (a 256-row tile owns both accumulators)
+        const uint32_t acc_use = MT == 2 ? (uint32_t)lt : (uint32_t)(lt >> 1);   // how often this buffer has been used
+        ok = ptx::mbar_wait(&acc_empty[buf], (acc_use & 1) ^ 1, abort_flag, p.dev_status);   // epilogue done with it
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t tmem_acc = tmem_base + (uint32_t)buf * S::kAccStride;
@@ -226,6 +233,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           for (int kk = 0; kk < kBK / 16; ++kk) {
             ptx::mma_ss(tmem_acc, ptx::smem_desc_advance(ad, kk * 32), ptx::smem_desc_advance(bd, kk * 32), idesc,
                         (kbk > kb0 || kk > 0) ? 1u : 0u);
+            if (MT == 2)   // rows 128..255 of the A stage against the same B tile, into the second accumulator
+              ptx::mma_ss(tmem_acc + S::kAccStride, ptx::smem_desc_advance(ad, kBM * kBK * 2 + kk * 32),
+                          ptx::smem_desc_advance(bd, kk * 32), idesc, (kbk > kb0 || kk > 0) ? 1u : 0u);
           }
           ptx::mma_commit(&empty[s]);     // frees the stage once these MMAs have read it
         }
@@ -245,17 +255,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       un.set(p, u);
       const int t = un.t, sp = un.sp;
       if (!tc.set(p, t)) continue;
-      const int buf = lt & 1;
+      const int buf = MT == 2 ? 0 : (lt & 1);
+      const uint32_t acc_use = MT == 2 ? (uint32_t)lt : (uint32_t)(lt >> 1);
       if (EPI == kEpiSim) {
         // inverse norms of this tile's kept rows; the four epilogue warps share them (named barrier 1)
         asm volatile("bar.sync 1, 128;" ::: "memory");          // everyone is done with the previous tile's values
         for (int j = et; j < BN; j += 128) ink_s[j] = (tc.n0 + j < tc.kb) ? p.inv_norm_kept[tc.k0 + tc.n0 + j] : 0.f;
         asm volatile("bar.sync 1, 128;" ::: "memory");
       }
-      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[buf], (lt >> 1) & 1, abort_flag, p.dev_status));
+      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[buf], acc_use & 1, abort_flag, p.dev_status));
       if (!ok) break;
       ptx::tc_fence_after_sync();
-      const uint32_t t_row = tmem_base + (uint32_t)buf * S::kAccStride + ((uint32_t)(quarter * 32) << 16);
+      uint32_t t_row = tmem_base + (uint32_t)buf * S::kAccStride + ((uint32_t)(quarter * 32) << 16);
+      int m_base = tc.m0;                                       // first row of the 128-row half in hand
       // A tile whose K range is cut into slices on different SMs: every unit writes its partial sums out
       // (column-major, so a warp's 32 rows are one 128-byte line); the unit that completes the tile (a
       // counter, left at zero again) adds the parts in the order of the K slices and runs the epilogue on
@@ -316,8 +328,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
       };
       if (!last) { ++lt; continue; }
+      // (a 256-row tile: the same epilogue once per 128-row half, each half in its own accumulator)
+#pragma unroll 1
+      for (int mh = 0; mh < MT; ++mh, t_row += S::kAccStride, m_base += kBM) {
       if (EPI == kEpiProj) {
-        const int grow = tc.m0 + row;
+        const int grow = m_base + row;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           float r[32];
@@ -339,7 +354,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       } else if (EPI == kEpiLinear) {
-        const int grow = tc.m0 + row;
+        const int grow = m_base + row;
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           float r[32];
@@ -365,7 +380,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       } else if (EPI == kEpiGateUp) {
-        const int grow = tc.m0 + row;
+        const int grow = m_base + row;
 #pragma unroll 1
         for (int c = 0; c < BN / 2; c += 32) {
           float g[32], up[32];
@@ -390,7 +405,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       } else {
-        const int m = tc.m0 + row;
+        const int m = m_base + row;
         const int g = tc.v0 + m;
         const bool active = m < tc.Vb && p.assign[g] < 0;     // a pruned token of this request
         const float inm = active ? p.inv_norm[g] : 0.f;
@@ -419,6 +434,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
               ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
           atomicMax(p.best + g, mine);
         }
+      }
       }
       if (split) { ++lt; continue; }                      // (its accumulator was released when the partial went out)
       // the accumulator may be overwritten once all four warps have read it
@@ -470,19 +486,31 @@ void plan_tail_split(const d3tom_ctx* ctx, GemmParams& p) {
   if (best_s > 1) { p.k_splits = best_s; p.full_tiles = tiles - rem; }
 }
 
-template <int BN, int EPI>
+// Measured main-loop cycles per 64-deep k-block with every SM busy: 780 for a 128 x 256 tile (its operands come out
+// of L2 at the rate all SMs together can get), 1060 for a 256 x 256 tile (tensor-bound: 8 MMAs of 128 cycles).
+constexpr double kCyclesM1 = 780.0, kCyclesM2 = 1060.0;
+
+// true when 256-row tiles finish the (rows x n_cols) layer sooner than the best 128-row tiling does
+bool prefer_two_m_tiles(const d3tom_ctx* ctx, int rows, int n_tiles_256, double cost_m1_in_667_units) {
+  const long long tiles2 = (long long)ceil_div(rows, 2 * kBM) * n_tiles_256;
+  const double rounds2 = (double)((tiles2 + ctx->sm_count - 1) / ctx->sm_count);
+  return rounds2 * kCyclesM2 < cost_m1_in_667_units * (kCyclesM1 / 667.0);
+}
+
+template <int BN, int EPI, int MT = 1>
 int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t s) {
-  if (EPI != kEpiSim) {
+  if (EPI != kEpiSim && MT == 1) {
     p.split_ws = ctx->gemm_split_ws; p.split_counters = ctx->gemm_split_counters;
     plan_tail_split(ctx, p);
   }
+  if (MT == 2) { p.k_splits = 1; p.full_tiles = p.m_tiles * p.n_tiles * p.batch; }   // whole tiles only
   const long long tiles = (long long)p.m_tiles * p.n_tiles * p.batch;
   const long long units = p.full_tiles + (tiles - p.full_tiles) * p.k_splits;
   if (units <= 0) return D3TOM_OK;
   const int grid = (int)(units < ctx->sm_count ? units : ctx->sm_count);          // persistent: one CTA per SM
-  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           GemmSmem<BN>::kBytes));
-  D3TOM_CUDA_TRY(ctx, launch_serialized(gemm_tc_kernel<BN, EPI>, grid, kGemmThreads, GemmSmem<BN>::kBytes, s, ta, tb, p));
+  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tc_kernel<BN, EPI, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           GemmSmem<BN, MT>::kBytes));
+  D3TOM_CUDA_TRY(ctx, launch_serialized(gemm_tc_kernel<BN, EPI, MT>, grid, kGemmThreads, GemmSmem<BN, MT>::kBytes, s, ta, tb, p));
   return D3TOM_OK;
 }
 
@@ -525,6 +553,13 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
+  if ((3 * D) % 256 == 0 && prefer_two_m_tiles(ctx, total, 3 * D / 256, best_cost)) {
+    r = make_tmap_bf16_2d(&ta, x, (uint64_t)total, (uint64_t)D, (uint64_t)D, 2 * kBM);
+    if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 256);
+    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+    p.m_tiles = ceil_div(total, 2 * kBM); p.n_tiles = 3 * D / 256;
+    return launch_gemm<256, kEpiProj, 2>(ctx, ta, tb, p, s);
+  }
   r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, (uint32_t)bn);
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
   p.n_tiles = 3 * D / bn;
@@ -554,6 +589,13 @@ int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* r
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
+  if (N % 256 == 0 && prefer_two_m_tiles(ctx, rows, N / 256, best_cost)) {
+    r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)K, (uint64_t)K, 2 * kBM);
+    if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, 256);
+    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+    p.m_tiles = ceil_div(rows, 2 * kBM); p.n_tiles = N / 256;
+    return launch_gemm<256, kEpiLinear, 2>(ctx, ta, tb, p, s);
+  }
   r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn);
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
   p.n_tiles = N / bn;
@@ -574,6 +616,16 @@ int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int 
   p.lin_out = static_cast<__nv_bfloat16*>(act); p.ld_out = m; p.up_row_offset = m; p.out_rows = rows;
   p.dev_status = ctx->dev_status;
   p.m_tiles = ceil_div(rows, kBM); p.n_tiles = m / 128; p.batch = 1; p.k_splits = 1;
+  {
+    const long long tiles1 = (long long)p.m_tiles * p.n_tiles;
+    const double cost1 = (double)((tiles1 + ctx->sm_count - 1) / ctx->sm_count) * 667.0;
+    if (prefer_two_m_tiles(ctx, rows, m / 128, cost1)) {
+      r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)D, (uint64_t)D, 2 * kBM);
+      if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+      p.m_tiles = ceil_div(rows, 2 * kBM);
+      return launch_gemm<256, kEpiGateUp, 2>(ctx, ta, tb, p, s);
+    }
+  }
   return launch_gemm<256, kEpiGateUp>(ctx, ta, tb, p, s);
 }
 
