@@ -486,9 +486,10 @@ void plan_tail_split(const d3tom_ctx* ctx, GemmParams& p) {
   if (best_s > 1) { p.k_splits = best_s; p.full_tiles = tiles - rem; }
 }
 
-// Measured main-loop cycles per 64-deep k-block with every SM busy: 780 for a 128 x 256 tile (its operands come out
-// of L2 at the rate all SMs together can get), 1060 for a 256 x 256 tile (tensor-bound: 8 MMAs of 128 cycles).
-constexpr double kCyclesM1 = 780.0, kCyclesM2 = 1060.0;
+// Measured main-loop cycles per 64 of K with every SM busy: 800 for a 128 x 256 tile (48 KB of operands: 61 B/clk
+// out of L2, what four 48 KB stages in flight yield at the load latency of about 2800 cycles), 1450 for a 256 x 256
+// tile (64 KB: 44 B/clk with three coarse 64 KB stages; 8 MMAs of 128 cycles would need 1024).
+constexpr double kCyclesM1 = 800.0, kCyclesM2 = 1450.0;
 
 // true when 256-row tiles finish the (rows x n_cols) layer sooner than the best 128-row tiling does
 bool prefer_two_m_tiles(const d3tom_ctx* ctx, int rows, int n_tiles_256, double cost_m1_in_667_units) {
