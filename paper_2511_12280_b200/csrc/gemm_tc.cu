@@ -486,16 +486,19 @@ void plan_tail_split(const d3tom_ctx* ctx, GemmParams& p) {
   if (best_s > 1) { p.k_splits = best_s; p.full_tiles = tiles - rem; }
 }
 
-// Measured main-loop cycles per 64 of K with every SM busy: 800 for a 128 x 256 tile (48 KB of operands: 61 B/clk
-// out of L2, what four 48 KB stages in flight yield at the load latency of about 2800 cycles), 1450 for a 256 x 256
-// tile (64 KB: 44 B/clk with three coarse 64 KB stages; 8 MMAs of 128 cycles would need 1024).
-constexpr double kCyclesM1 = 800.0, kCyclesM2 = 1450.0;
-
-// true when 256-row tiles finish the (rows x n_cols) layer sooner than the best 128-row tiling does
-bool prefer_two_m_tiles(const d3tom_ctx* ctx, int rows, int n_tiles_256, double cost_m1_in_667_units) {
-  const long long tiles2 = (long long)ceil_div(rows, 2 * kBM) * n_tiles_256;
-  const double rounds2 = (double)((tiles2 + ctx->sm_count - 1) / ctx->sm_count);
-  return rounds2 * kCyclesM2 < cost_m1_in_667_units * (kCyclesM1 / 667.0);
+// Which tile shape finishes a dense layer sooner, from measured main-loop cycles per 64 of K (projection timings at
+// 128 .. 4288 rows).  128 x 256 tiles: 850 per full round over the SMs (48 KB of operands per k-block: what the SMs
+// together can pull out of L2), and 150 + 3.9 r for a last round of r tiles, which runs faster per tile because
+// fewer SMs share L2.  256 x 256 tiles: 1450 per full round (64 KB per k-block in three 64 KB stages: bound by the
+// load latency of one SM, so a round of few tiles is no cheaper), 900 + 3.5 r for the last round.  The larger tile
+// wins when it saves a round of the smaller one.
+bool prefer_two_m_tiles(const d3tom_ctx* ctx, int rows, int n_tiles_256) {
+  const int sms = ctx->sm_count;
+  const long long t1 = (long long)ceil_div(rows, kBM) * n_tiles_256, t2 = (long long)ceil_div(rows, 2 * kBM) * n_tiles_256;
+  const double r1 = (double)(t1 % sms), r2 = (double)(t2 % sms);
+  const double cost1 = 850.0 * (double)(t1 / sms) + (r1 > 0 ? 150.0 + 3.9 * r1 : 0.0);
+  const double cost2 = 1450.0 * (double)(t2 / sms) + (r2 > 0 ? 900.0 + 3.5 * r2 : 0.0);
+  return cost2 < 0.97 * cost1;
 }
 
 template <int BN, int EPI, int MT = 1>
@@ -554,7 +557,7 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  if ((3 * D) % 256 == 0 && prefer_two_m_tiles(ctx, total, 3 * D / 256, best_cost)) {
+  if ((3 * D) % 256 == 0 && prefer_two_m_tiles(ctx, total, 3 * D / 256)) {
     r = make_tmap_bf16_2d(&ta, x, (uint64_t)total, (uint64_t)D, (uint64_t)D, 2 * kBM);
     if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 256);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
@@ -590,7 +593,7 @@ int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* r
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  if (N % 256 == 0 && prefer_two_m_tiles(ctx, rows, N / 256, best_cost)) {
+  if (N % 256 == 0 && prefer_two_m_tiles(ctx, rows, N / 256)) {
     r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)K, (uint64_t)K, 2 * kBM);
     if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, 256);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
@@ -618,9 +621,7 @@ int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int 
   p.dev_status = ctx->dev_status;
   p.m_tiles = ceil_div(rows, kBM); p.n_tiles = m / 128; p.batch = 1; p.k_splits = 1;
   {
-    const long long tiles1 = (long long)p.m_tiles * p.n_tiles;
-    const double cost1 = (double)((tiles1 + ctx->sm_count - 1) / ctx->sm_count) * 667.0;
-    if (prefer_two_m_tiles(ctx, rows, m / 128, cost1)) {
+    if (prefer_two_m_tiles(ctx, rows, m / 128)) {
       r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)D, (uint64_t)D, 2 * kBM);
       if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
       p.m_tiles = ceil_div(rows, 2 * kBM);
