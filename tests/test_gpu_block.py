@@ -56,6 +56,14 @@ def test_linear_and_ffn_bf16_long_k_few_tiles_cut_into_k_slices():
     run_ffn(300, 4096, 256, "bf16", seed=4)
 
 
+def test_linear_and_ffn_bf16_shapes_that_take_256_row_tiles():
+    # 1500 rows x 48 column tiles: 256-row CTA tiles finish sooner than 128-row ones here (two rounds over the SMs
+    # instead of four), for the linear layer and for the gate/up pass; the last tile has 220 of 256 rows
+    run_linear(1500, 64, 12288, "bf16", residual=True, seed=5)
+    run_linear(1500, 128, 12288, "bf16", residual=False, seed=6)
+    run_ffn(1500, 128, 6144, "bf16", seed=7)
+
+
 def test_linear_fp32_odd_sizes():
     run_linear(70, 50, 45, "fp32", residual=True)
     run_linear(33, 7, 3, "fp32", residual=False)
