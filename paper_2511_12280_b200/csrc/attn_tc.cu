@@ -393,7 +393,7 @@ int launch(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
                                            AttnSmem<DH>::kBytes));
   AttnArgs k = a;
   k.nqb = ceil_div(a.max_seqlen, 2 * kTile);
-  const int items = a.H * k.nqb, sms = ctx->sm_count;
+  const int items = a.H * k.nqb, sms = ctx->sm_count > 0 ? ctx->sm_count : 1;
   k.split_from = items;
   if (a.B == 1) {                                   // (with one request the row count is known here)
     const int rest = items % sms;

@@ -33,9 +33,10 @@ constexpr int kMaxDevices = 64;
 std::mutex g_mutex;
 unsigned char* g_base[kMaxDevices];      // device address of g_static_scratch on each device, once looked up
 int g_major[kMaxDevices];
+int g_sm_count[kMaxDevices];             // multiprocessors of each device (the attention launcher shapes its grid by it)
 
 // Looks up (once per device) the device address of the array on the CURRENT device.
-int static_scratch_base(int* device_out, unsigned char** base_out) {
+int static_scratch_base(int* device_out, unsigned char** base_out, int* sm_count_out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return D3TOM_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_mutex);
@@ -44,6 +45,9 @@ int static_scratch_base(int* device_out, unsigned char** base_out) {
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return D3TOM_ERR_CUDA;
     g_major[dev] = major;
     if (major != 10) return D3TOM_ERR_UNSUPPORTED;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return D3TOM_ERR_CUDA;
+    g_sm_count[dev] = sms;
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
       (void)cudaGetLastError();
@@ -54,6 +58,7 @@ int static_scratch_base(int* device_out, unsigned char** base_out) {
   if (g_major[dev] != 10) return D3TOM_ERR_UNSUPPORTED;
   *device_out = dev;
   *base_out = g_base[dev];
+  *sm_count_out = g_sm_count[dev];
   return D3TOM_OK;
 }
 
@@ -87,15 +92,16 @@ extern "C" int d3tom_attn_importance_static(d3tom_dtype dt, int heads, int head_
     return D3TOM_ERR_WORKSPACE;
   if (total_tokens == 0 || max_seqlen == 0) return D3TOM_OK;
 
-  int dev = -1;
+  int dev = -1, sms = 0;
   unsigned char* base = nullptr;
-  int st = static_scratch_base(&dev, &base);
+  int st = static_scratch_base(&dev, &base, &sms);
   if (st != D3TOM_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 
   // a context that lives on the host stack and only points into the array: nothing is allocated
   d3tom_ctx c = {};
   c.device = dev;
+  c.sm_count = sms;
   c.lim.max_total_tokens = total_tokens; c.lim.max_batch = B; c.lim.heads = heads; c.lim.head_dim = head_dim;
   c.lim.max_deciders = (int)nd; c.lim.max_visual_per_request = max_visual;
   c.vis_stride = (int)vis_stride;

@@ -1,12 +1,16 @@
 """d3tom_attn_importance_static, the entry point for hosts that may not allocate
 device memory (no context; scratch in a fixed array of the library image), must
-give what d3tom_attn_importance gives.  Two calls in a row on different
-problems share that array, so the second one also shows that nothing left over
-from the first leaks into the results.  This file is collected last on purpose."""
+give what d3tom_attn_importance gives, and what the CPU oracle gives.  Calls in
+a row on different problems share that array, so each later one also shows that
+nothing left over from the one before leaks into the results.  Batches of one
+request take the launcher's own grid shapes (single-tile CTAs for a tiny grid or
+for an incomplete last wave), so both of those are among the problems.  This
+file is collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import d3tom_oracle as orc
 from paper_2511_12280_b200 import binding as B_
 from paper_2511_12280_b200 import workload as wl
 
@@ -21,7 +25,12 @@ def _problems():
     b = wl.make_workload("static_b", "bf16", 2, 64, 22, 8,
                          [dict(V=131, P=9, O=20, n_dec=2, r=0.3), dict(V=90, P=2, O=6, n_dec=0, r=0.3),
                           dict(V=300, P=1, O=3, n_dec=1, r=0.3)])
-    return [a, b]
+    # one request, few work items: every 128-row tile becomes a CTA of its own
+    c = wl.make_workload("static_c", "bf16", 4, 128, 23, 8, [dict(V=200, P=20, O=30, n_dec=6, r=0.3)])
+    # one request at the LLaDA-8B shape (the C1 configuration): 160 work items on 148 SMs, so the items of the
+    # incomplete last wave are cut in two
+    d = wl.config("C1")
+    return [a, b, c, d]
 
 
 def _run_both(w):
@@ -55,6 +64,16 @@ def test_static_entry_point_matches_the_context_one_on_two_calls_in_a_row():
         assert np.isfinite(gi).all()
         assert (np.abs(gi - wi) <= 1e-4 * np.abs(wi) + 1e-7).all()
         assert torch.equal(imp, want_imp)
+        # and against the oracle itself, not only against the other entry point
+        q, k, v = pu.f64(w.q_for()), pu.f64(w.k), pu.f64(w.v)
+        scale = 1.0 / np.sqrt(w.dh)
+        want = orc.round_storage(orc.attention(q, k, v, w.cu_seqlens, scale), w.dtype)
+        pu.assert_close(pu.f64(out), want, w.dtype, "static attention output against the oracle")
+        dec = np.concatenate([np.asarray(d, np.int64) for d in w.decider_pos])
+        S = orc.importance(q, k, w.cu_seqlens, w.n_visual, dec, w.cu_deciders(), scale)
+        for b in range(w.B):
+            g = gi[w.cu_vis[b]:w.cu_vis[b + 1]]
+            assert (np.abs(g - S[b]) <= 1e-4 * np.abs(S[b]) + 1e-7 * len(w.decider_pos[b]) * w.H).all()
 
 
 def test_static_entry_point_rejects_sizes_beyond_its_array():
