@@ -33,10 +33,11 @@ select_kernel(const float* __restrict__ importance, const int32_t* __restrict__ 
   grid_dependency_enter();
   const int b = blockIdx.x;
   const int v0 = cu_vis[b], V = cu_vis[b + 1] - v0;
-  const int k = keep_count[b];
   const float* sc = importance + v0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (V <= 0) return;
+  int k = keep_count[b];
+  k = k < 0 ? 0 : (k > V ? V : k);          // as select_reg_kernel: a count outside [0, V] cannot leave the segment
 
   if (kKeysInSmem) {
     for (int j = tid; j < V; j += kThreads) keys_s[j] = ordered_key(sc[j]);
@@ -48,7 +49,7 @@ select_kernel(const float* __restrict__ importance, const int32_t* __restrict__ 
   // ---- radix select of the k-th largest key ----
   uint32_t mask = 0u;
   const int v_round = ((V + 31) / 32) * 32;
-  for (int pass = 0; pass < 4; ++pass) {
+  for (int pass = 0; pass < (k > 0 ? 4 : 0); ++pass) {   // k = 0: nothing is kept, there is no key of rank k
     const int shift = 24 - 8 * pass;
     for (int d = tid; d < 256; d += kThreads) sh.hist[d] = 0u;
     __syncthreads();
@@ -94,7 +95,7 @@ select_kernel(const float* __restrict__ importance, const int32_t* __restrict__ 
     __syncthreads();
   }
   const uint32_t T = sh.prefix;          // key of rank k
-  const unsigned need_eq = sh.remaining; // how many keys == T are kept (lowest indices first)
+  const unsigned need_eq = k > 0 ? sh.remaining : 0u; // how many keys == T are kept (lowest indices first)
 
   // ---- ordered output pass ----
   if (tid == 0) sh.carry = 0u;           // packed running totals: (greater << 16 | equal) per chunk, 32-bit each below
@@ -107,7 +108,7 @@ select_kernel(const float* __restrict__ importance, const int32_t* __restrict__ 
     const int j = base + tid;
     uint32_t key = 0u;
     bool gt = false, eq = false;
-    if (j < V) { key = key_at(j); gt = key > T; eq = key == T; }
+    if (j < V && k > 0) { key = key_at(j); gt = key > T; eq = key == T; }
     // packed per-thread counts: high 16 bits greater, low 16 bits equal (chunk <= 1024)
     unsigned val = (gt ? 0x10000u : 0u) | (eq ? 1u : 0u);
     unsigned incl = val;

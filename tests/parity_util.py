@@ -41,16 +41,56 @@ def assert_close(got, want, dtype, what):
     return float(err.max())
 
 
+GUARD_ROWS = 5          # slack rows behind every output buffer; nothing may write there
+POISON_INT, POISON_U8 = -1, 0xAB
+
+
+def _output_buffers(step):
+    """(name, tensor, rows the step may write) of every buffer a step writes."""
+    bufs = [("attn_out", step.attn_out, step.total), ("importance", step.importance, step.total_vis),
+            ("kept_idx", step.kept_idx, step.total_kept), ("keep_mask", step.keep_mask, step.total_vis),
+            ("assign", step.assign, step.total_vis), ("member_count", step.member_count, step.total_kept),
+            ("src_of_dst", step.src_of_dst, step.total_out), ("hidden_out", step.hidden_out, step.total_out)]
+    if step.n_post:
+        bufs += [("q2", step.q2, step.total_out), ("k2", step.k2, step.total_out), ("v2", step.v2, step.total_out)]
+        bufs += [("layer_out%d" % l, t, step.total_out) for l, t in enumerate(step.layer_out)]
+    return bufs
+
+
+def _poison_value(t):
+    return float("nan") if t.dtype.is_floating_point else (POISON_U8 if t.dtype == torch.uint8 else POISON_INT)
+
+
+def poison_outputs(step):
+    """Fills every output buffer (slack rows included) with NaN / -1 / 0xAB, so that an element the
+    kernels forget to write cannot pass by holding an earlier run's correct value."""
+    for _, t, _ in _output_buffers(step):
+        t.fill_(_poison_value(t))
+
+
+def assert_guard_rows_untouched(step):
+    """The rows behind the part of each buffer that this problem owns still hold the poison."""
+    for name, t, used in _output_buffers(step):
+        tail = t[used:]
+        assert tail.shape[0] >= GUARD_ROWS, name
+        if t.dtype.is_floating_point:
+            assert bool(torch.isnan(tail).all()), "%s: a kernel wrote past row %d" % (name, used)
+        else:
+            assert bool((tail == _poison_value(t)).all()), "%s: a kernel wrote past element %d" % (name, used)
+
+
 def make_step(w, n_post=None, mode=B_.AGG_MEAN, sim_debug=True, decider_pos=None, keep_count=None) -> MergeLayerStep:
+    """A step whose buffers are GUARD_ROWS rows longer than the problem and poisoned."""
     n_post = len(w.w_post) if n_post is None else n_post
     decider_pos = w.decider_pos if decider_pos is None else decider_pos
     if keep_count is None:
         keep_count = [B_.d3tom_keep_count(v, r) if len(d) else v
                       for v, r, d in zip(w.n_visual, w.keep_ratio, decider_pos)]
     total = int(w.cu_seqlens[-1])
-    step = MergeLayerStep(w.H, w.dh, w.torch_dtype, total, w.B, sum(len(d) for d in decider_pos),
+    step = MergeLayerStep(w.H, w.dh, w.torch_dtype, total + GUARD_ROWS, w.B, sum(len(d) for d in decider_pos),
                           max(w.n_visual), n_post=n_post, mode=mode, sim_debug=sim_debug)
     step.set_problem(w.n_visual, w.n_prompt, w.n_resp, decider_pos, keep_count)
+    poison_outputs(step)
     return step
 
 
@@ -69,6 +109,7 @@ def check_step(w, mode=B_.AGG_MEAN, full_attention=True, n_sample_rows=48, decid
     step.run(q, k, v, w_post)
     torch.cuda.synchronize()
     assert step.ctx.device_status() == 0, "device status word reports a kernel-side problem"
+    assert_guard_rows_untouched(step)
 
     rep = {}
     H, dh, D, dt = w.H, w.dh, w.D, w.dtype
@@ -79,6 +120,7 @@ def check_step(w, mode=B_.AGG_MEAN, full_attention=True, n_sample_rows=48, decid
 
     # ---- (0) attention output H~
     attn_gpu = f64(step.attn_out[:total])
+    assert np.isfinite(attn_gpu).all(), "attention output has unwritten (poisoned) elements"
     if full_attention:
         want = orc.round_storage(orc.attention(qn, kn, vn, cu, scale), dt)
         rep["attn"] = assert_close(attn_gpu, want, dt, "attention output")
@@ -178,6 +220,7 @@ def check_step(w, mode=B_.AGG_MEAN, full_attention=True, n_sample_rows=48, decid
         for l in range(step.n_post):
             wl = f64(w.w_post[l])
             got = f64(step.layer_out[l][:step.total_out])
+            assert np.isfinite(got).all(), "post-merge layer %d has unwritten (poisoned) elements" % l
             if full_attention:
                 want = orc.post_layer(x, wl, step.cu_out_h, H, dt)
                 rep["post%d" % l] = assert_close(got, want, dt, "post-merge layer %d" % l)

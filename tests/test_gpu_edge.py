@@ -45,8 +45,8 @@ def test_many_rows_fp32_take_the_streaming_aggregation():
     # serving config); narrow rows keep the oracle cheap
     reqs = [dict(V=3000, P=40, O=12, n_dec=3, r=0.8), dict(V=2600, P=9, O=8, n_dec=2, r=0.7)]
     w = wl.make_workload("rows", "fp32", 2, 32, 13, 16, reqs, post_layers=0)
-    pu.check_step(w, full_attention=False, n_sample_rows=8)
-    pu.check_step(w, mode=B_.AGG_SUM, full_attention=False, n_sample_rows=8)
+    pu.check_step(w)
+    pu.check_step(w, mode=B_.AGG_SUM)
 
 
 def test_single_request_single_tile_ctas_with_deciders():
@@ -61,6 +61,7 @@ def test_kept_set_larger_than_the_shared_memory_counters():
     # more than 12288 kept tokens in one request: the member counters live in global memory, the bitmap of a
     # sorting warp spans 13000 positions, and select stages 13000 keys
     w = small(H=1, dh=64, reqs=[dict(V=13000, P=8, O=8, n_dec=3, r=0.97)], post=0)
+    # (attention on sampled rows: the oracle's full 13016 x 13016 fp64 matrix would take several GB of host memory)
     pu.check_step(w, full_attention=False, n_sample_rows=6)
 
 
@@ -125,11 +126,12 @@ def run_select(scores_list, ks):
     dev = torch.device("cuda", 0)
     imp = torch.as_tensor(np.concatenate(scores_list).astype(np.float32), device=dev)
     t = lambda a: torch.as_tensor(np.asarray(a, np.int32), device=dev)
-    kept = torch.full((int(cu_kept[-1]),), -7, dtype=torch.int32, device=dev)
-    mask = torch.full((int(cu_vis[-1]),), 9, dtype=torch.uint8, device=dev)
+    kept = torch.full((int(cu_kept[-1]) + 4,), -7, dtype=torch.int32, device=dev)     # 4 guard elements each
+    mask = torch.full((int(cu_vis[-1]) + 4,), 9, dtype=torch.uint8, device=dev)
     ctx.d3tom_select(imp, t(cu_vis), t(ks), t(cu_kept), B, max(V), kept, mask)
     torch.cuda.synchronize()
     kept, mask = kept.cpu().numpy(), mask.cpu().numpy()
+    assert (kept[cu_kept[-1]:] == -7).all() and (mask[cu_vis[-1]:] == 9).all()
     for b in range(B):
         want = orc.select(scores_list[b].astype(np.float32), ks[b])
         assert np.array_equal(kept[cu_kept[b]:cu_kept[b + 1]], want), b
@@ -151,6 +153,11 @@ def test_select_adversarial_inputs():
     y = np.array([np.nextafter(base, np.float32(1), dtype=np.float32) if i % 3 == 0 else base for i in range(2000)], np.float32)
     run_select([y], [700])
     run_select([rng.random(70000)], [12345])             # larger than the shared-memory staging
+    # between 8192 and 40960 tokens per request the keys are staged in shared memory; a keep count of 0 (nothing
+    # kept: all-zero mask, no index written) and one of |V| (everything kept) in the same launch
+    run_select([rng.random(20000), rng.integers(0, 3, 9000) / 4.0, rng.random(8193)], [5000, 0, 8193])
+    run_select([rng.random(50000), rng.random(100)], [0, 100])
+    run_select([rng.random(3000), rng.random(100)], [0, 7])                 # keys in registers, keep count 0
 
 
 def test_host_made_failures_return_status_codes():
@@ -163,7 +170,7 @@ def test_host_made_failures_return_status_codes():
     s = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
     P = lambda t: ctypes.c_void_p(t.data_ptr())
     # workspace limits
-    assert lib.d3tom_attn_varlen(h, B_.BF16, P(q), P(k), P(v), P(step.cu_seqlens), step.nB, step.total + 1,
+    assert lib.d3tom_attn_varlen(h, B_.BF16, P(q), P(k), P(v), P(step.cu_seqlens), step.nB, step.total + pu.GUARD_ROWS + 1,
                                  step.max_seqlen, 0.1, P(step.attn_out), s) == B_.ERR_WORKSPACE
     assert lib.d3tom_attn_varlen(h, B_.BF16, P(q), P(k), P(v), P(step.cu_seqlens), step.nB + 1, step.total,
                                  step.max_seqlen, 0.1, P(step.attn_out), s) == B_.ERR_WORKSPACE

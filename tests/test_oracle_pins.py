@@ -327,6 +327,44 @@ def test_post_layer_is_projection_then_attention():
     assert np.array_equal(y, orc.round_bf16(orc.attention(q, k, v, [0, 4, n], 1 / math.sqrt(dh))))
 
 
+def test_proj_qkv_hand_computed_two_rows():
+    # every number below is worked out by hand from Q = X W_q^T, K = X W_k^T, V = X W_v^T with
+    # W = [W_q; W_k; W_v] stored [out, in]: rows 0-1 -> Q, rows 2-3 -> K, rows 4-5 -> V
+    x = np.array([[1.0, 2.0], [3.0, -1.0]])
+    w = np.array([[1.0, 2.0], [3.0, 4.0],        # W_q
+                  [-1.0, 0.5], [0.0, -2.0],      # W_k
+                  [0.5, 0.5], [2.0, -1.0]])      # W_v
+    for H in (1, 2):                             # one head of width 2, two heads of width 1: same numbers, other shape
+        q, k, v = orc.proj_qkv(x, w, H, "bf16")
+        assert q.shape == k.shape == v.shape == (2, H, 2 // H)
+        assert q.reshape(2, 2).tolist() == [[5.0, 11.0], [1.0, 5.0]]
+        assert k.reshape(2, 2).tolist() == [[0.0, -4.0], [-3.5, 2.0]]
+        assert v.reshape(2, 2).tolist() == [[1.5, 0.0], [1.0, 7.0]]
+    q2 = orc.proj_qkv(x, w, 2, "bf16")[0]
+    assert q2[0, 1, 0] == 11.0 and q2[1, 0, 0] == 1.0          # head h is column h when dh = 1
+    # one product that the storage type changes: 1 + 3 * 2^-9 lies between the bf16 neighbours 1 and 1 + 2^-7
+    # (closer to the upper one); fp32 holds it exactly
+    xr = np.array([[1.0, 1.0]])
+    wr = np.tile(np.array([[1.0, 3.0 / 512.0]]), (6, 1))
+    assert orc.proj_qkv(xr, wr, 1, "bf16")[1][0, 0, 0] == 1.0078125
+    assert orc.proj_qkv(xr, wr, 1, "fp32")[1][0, 0, 0] == 1.005859375
+    # an exact tie (1 + 2^-8) goes to the even neighbour, 1
+    wt = np.tile(np.array([[1.0, 1.0 / 256.0]]), (6, 1))
+    assert orc.proj_qkv(xr, wt, 1, "bf16")[2][0, 0, 0] == 1.0
+
+
+def test_post_layer_with_zero_query_weights_averages_the_values():
+    # W_q = 0 makes every score 0, the softmax uniform, and the layer's output the mean of the request's V rows:
+    # with the hand-computed V = [[1.5, 0], [1, 7]] of the case above that is [1.25, 3.5] for both rows
+    x = np.array([[1.0, 2.0], [3.0, -1.0]])
+    w = np.array([[0.0, 0.0], [0.0, 0.0], [-1.0, 0.5], [0.0, -2.0], [0.5, 0.5], [2.0, -1.0]])
+    y = orc.post_layer(x, w, [0, 2], 1, "bf16")
+    assert y.tolist() == [[1.25, 3.5], [1.25, 3.5]]
+    # two requests of one row each: every row attends to itself only, the output is its own V row
+    y = orc.post_layer(x, w, [0, 1, 2], 1, "bf16")
+    assert y.tolist() == [[1.5, 0.0], [1.0, 7.0]]
+
+
 # ------------------------------------------------------------------ schedule + FLOP tables
 def test_schedule_endpoints_mean_direction():
     T = 64
