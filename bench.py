@@ -8,18 +8,28 @@ merge-layer attention + importance map, select, merge (similarity, aggregation,
 compaction) and the post-merge layers (projection + ragged attention each).
 The default workload is C2, the LLaDA-8B-shaped configuration with thousands of
 visual tokens (4096 visual + 128 prompt + 64 response tokens, keep ratio 0.25,
-3 post-merge layers).  One JSON line is printed by rank 0.
+3 post-merge layers).  One JSON line is printed by rank 0.  Beside the step time
+of the chosen configuration it carries
 
-With N > 1 (launched by torch.distributed.run) every rank processes its own
-request of the same shape: the path shards by request, with no collective on
-the data path; the only communication is the barrier and the max-over-ranks of
-the timing.
+  roofline      the dominant kernel (merge-layer attention) against the measured tensor peak
+  kernels       every kernel of the step: device time inside running steps, algorithmic work,
+                fraction of the nominal, measured-burst and measured-sustained peaks
+  configs       step time, attention fraction and end-to-end time of the other configurations
+  cpu_baseline  the CPU oracle timed on one whole step of the same workload
+  e2e           the same step fed from pinned host memory, result copied back
+
+With N > 1 every rank processes its own request batch of the same shape: the
+path shards by request with no collective on the data path; the only
+communication is the barrier and the max-over-ranks of the timing.  Launched
+under torch.distributed.run the ranks come from the environment; launched
+plainly with --gpus N > 1 this script starts the N ranks itself.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -38,10 +48,12 @@ WORKLOAD_TEXT = {
           "one more decider per step, keep ratio 0.5 -> 0 (mean 0.25), 3 post-merge layers; a step = one denoising step",
     "C4": "C4: 8 ragged requests, 1024-4096 visual tokens each, 32 heads x 128, keep in {0.1,0.25,0.5}, 3 post-merge layers",
 }
-# DRAM bytes of one launch of the dominant kernel from the committed ncu capture (null for configs not captured,
-# and to be reset to null whenever attn_tc.cu changes after the capture)
-ATTN_TRAFFIC_BYTES = {"C2": 164.8e6}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the committed ncu
+# capture; null for configurations not captured, and null whenever attn_tc.cu has changed since the capture
+ATTN_TRAFFIC_BYTES = {"C2": None}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+REFERENCE_BUDGET_S = 240.0          # the CPU arm stops adding steps once they would not fit this
 
 
 def load_peaks():
@@ -125,58 +137,54 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ oracle timing
-def oracle_step_sample(w, heads=2, row_frac=8, decider_pos=None, keep=None):
-    """Times the CPU oracle, as it stands, on a bounded sample of one step of
-    workload ``w`` and extrapolates linearly to the full step:
-    attention and importance on ``heads`` of the H heads (x H/heads), select and
-    merge in full, one post-merge layer with its projection on 1/row_frac of the
-    rows (x row_frac) and its attention on ``heads`` heads (x H/heads), times the
-    number of post-merge layers.  Returns (seconds per full step, description)."""
+def oracle_inputs(w, decider_pos=None):
+    """The step's inputs as float64 arrays (conversion is not part of the timed oracle step)."""
+    import torch
+    decider_pos = w.decider_pos if decider_pos is None else decider_pos
+    q = w.q_for(decider_pos).to(dtype=torch.float64).numpy()
+    k = w.k.double().numpy()
+    v = w.v.double().numpy()
+    w_post = [x.double().numpy() for x in w.w_post]
+    return q, k, v, w_post
+
+
+def oracle_step(w, inputs, decider_pos=None, keep=None):
+    """One WHOLE step of workload ``w`` on the CPU oracle as it stands, nothing sampled or extrapolated:
+    attention over every head, importance, select, merge (MEAN) and every post-merge layer.
+    Returns (seconds, seconds per part)."""
     from oracle import d3tom_oracle as orc
+    q, k, v, w_post = inputs
     H, dh = w.H, w.dh
-    hs = min(heads, H)
     scale = 1.0 / np.sqrt(dh)
     cu = w.cu_seqlens
     decider_pos = w.decider_pos if decider_pos is None else decider_pos
-    q = w.q_for(decider_pos).to(dtype=__import__("torch").float64).numpy()
-    k = w.k.double().numpy()
-    v = w.v.double().numpy()
     dec = np.concatenate([np.asarray(d, np.int64) for d in decider_pos])
     t = {}
     t0 = time.perf_counter()
-    out_h = orc.attention(q[:, :hs], k[:, :hs], v[:, :hs], cu, scale)
-    t["attn"] = (time.perf_counter() - t0) * H / hs
+    hidden = orc.round_storage(orc.attention(q, k, v, cu, scale), w.dtype)
+    t["attn"] = time.perf_counter() - t0
     t0 = time.perf_counter()
-    S = orc.importance(q[:, :hs], k[:, :hs], cu, w.n_visual, dec, w.cu_deciders(decider_pos), scale)
-    t["importance"] = (time.perf_counter() - t0) * H / hs
+    S = orc.importance(q, k, cu, w.n_visual, dec, w.cu_deciders(decider_pos), scale)
+    t["importance"] = time.perf_counter() - t0
     t0 = time.perf_counter()
     if keep is None:
-        keep = [orc.keep_count(w.n_visual[b], w.keep_ratio[b]) for b in range(w.B)]
+        keep = [orc.keep_count(w.n_visual[b], w.keep_ratio[b]) if len(decider_pos[b]) else w.n_visual[b]
+                for b in range(w.B)]
     kept = [orc.select(S[b].astype(np.float32), keep[b]) for b in range(w.B)]
     t["select"] = time.perf_counter() - t0
-    hidden = np.zeros((q.shape[0], H * dh))
-    hidden[:, :hs * dh] = out_h
-    hidden = orc.round_storage(hidden, w.dtype)
     t0 = time.perf_counter()
     res = orc.merge(hidden, cu, w.n_visual, kept, orc.MEAN, w.dtype)
     t["merge"] = time.perf_counter() - t0
-    t["post"] = 0.0
-    if w.w_post:
-        x = res["hidden_out"]
-        wq = w.w_post[0].double().numpy()
-        n_sub = max(1, x.shape[0] // row_frac)
-        t0 = time.perf_counter()
-        orc.proj_qkv(x[:n_sub], wq, H, w.dtype)
-        t_proj = (time.perf_counter() - t0) * x.shape[0] / n_sub
-        qq = x.reshape(x.shape[0], H, dh)[:, :hs]
-        t0 = time.perf_counter()
-        orc.attention(qq, qq, qq, res["cu_seqlens_out"], scale)
-        t_att = (time.perf_counter() - t0) * H / hs
-        t["post"] = (t_proj + t_att) * len(w.w_post)
-    desc = ("oracle on %d of %d heads for attention/importance (x%d), select+merge in full, one post-merge layer "
-            "(projection on 1/%d of the rows, attention on %d heads) x%d layers; extrapolated linearly"
-            % (hs, H, H // hs, row_frac, hs, len(w.w_post)))
-    return sum(t.values()), desc, t
+    t0 = time.perf_counter()
+    x = res["hidden_out"]
+    for wl_ in w_post:
+        x = orc.post_layer(x, wl_, res["cu_seqlens_out"], H, w.dtype)
+    t["post"] = time.perf_counter() - t0
+    return sum(t.values()), t
+
+
+ORACLE_SAMPLE_TEXT = ("one whole step of the workload on the NumPy/fp64 oracle as it stands: attention over all heads, "
+                      "importance, select, merge (mean) and all post-merge layers; nothing sampled or extrapolated")
 
 
 def blas_threads():
@@ -188,7 +196,167 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def block_timings(step, w, w_post0, q, k, v, dev, timed, reps):
+def schedule_middle(w):
+    """Schedule config: decider list and keep count of the middle denoising step (the oracle's sampled step)."""
+    from oracle import d3tom_oracle as orc
+    sm = w.T // 2
+    a_min = 2.0 * (1.0 - w.mean_keep_ratio) - 1.0
+    return sm, dict(decider_pos=w.step_deciders(sm),
+                    keep=[orc.keep_count(w.n_visual[0], 1.0 - orc.schedule_alpha(sm, w.T, a_min, 1.0))])
+
+
+def reference_arm(args, config):
+    """The CPU oracle as the reference arm: every step is one whole oracle step of the workload."""
+    from paper_2511_12280_b200 import workload as wl
+    w = wl.config(args.config)
+    config["requests_per_gpu"] = w.B
+    kw = {}
+    if w.T:        # the schedule config is timed at its middle step
+        sm, kw = schedule_middle(w)
+        config["sampled_step"] = sm
+    inputs = oracle_inputs(w, kw.get("decider_pos"))
+    times, parts = [], {}
+    t_start = time.perf_counter()
+    warm_left, steps_timed, warm_done = args.warmup, 0, 0
+    while steps_timed < args.steps:
+        sec, parts = oracle_step(w, inputs, **kw)
+        if warm_left > 0:
+            warm_left -= 1
+            warm_done += 1
+        else:
+            times.append(sec)
+            steps_timed += 1
+        elapsed = time.perf_counter() - t_start
+        per = elapsed / (warm_done + steps_timed)
+        if elapsed + per > REFERENCE_BUDGET_S:          # the next step would not fit: stop here
+            if not times:                               # not even one timed step yet: the last warm-up step is the sample
+                times.append(sec)
+                steps_timed = 1
+                warm_done -= 1
+            break
+    us = float(np.mean(times)) * 1e6
+    line = {"impl": "reference", "metric": "merge_layer_step_us", "value": us, "unit": "us", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+            "steps_timed": steps_timed, "warmup_done": warm_done,
+            "step_us_median": float(np.median(times)) * 1e6, "step_us_min": float(np.min(times)) * 1e6,
+            "cpu_baseline": {"value": us, "unit": "us", "cores": blas_threads(), "kind": "oracle",
+                             "sample": ORACLE_SAMPLE_TEXT, "steps_timed": steps_timed, "extrapolated": False},
+            "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "breakdown_s": parts}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------ N ranks from a plain launch
+def spawn_ranks(args):
+    """`python bench.py --gpus N` with N > 1 and no launcher around it: start the N ranks (one per GPU, rendezvous on
+    127.0.0.1) with torch.distributed.run and pass their output through."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+# ------------------------------------------------------------------------------------------ per-kernel device times
+def step_kernel_labels(step):
+    """Kernels of one run() in launch order, as (label, substring its kernel name must contain)."""
+    seq = [("attn_merge_layer", "attn_"), ("importance_finish", "importance_finish"), ("select", "select"),
+           ("prepare_rows", "prepare_rows")]
+    if step.total_out < step.total:
+        seq.append(("similarity_gemm", "gemm_tc"))
+    seq += [("members", "members"), ("aggregate_compact", "aggregate")]
+    for _ in range(step.n_post):
+        seq += [("proj_qkv", "gemm_tc"), ("attn_post", "attn_")]
+    return seq
+
+
+def kernel_work(step, q):
+    """Algorithmic work of every kernel of the step: ("tensor", flops) or ("hbm", bytes)."""
+    D, H, es = step.D, step.H, q.element_size()
+    V, K = step.n_visual_h, step.keep_h
+    n_dec = [int(step.cu_dec_h[b + 1] - step.cu_dec_h[b]) for b in range(step.nB)]
+    tv, tk = sum(V), sum(K)
+    return {
+        "attn_merge_layer": ("tensor", sum(4.0 * n * n * D for n in step.seqlens_h)),
+        "importance_finish": ("hbm", sum(4.0 * H * d * v for d, v in zip(n_dec, V)) + 4.0 * tv),
+        "select": ("hbm", 4.0 * tv + 4.0 * tk + tv),
+        "prepare_rows": ("hbm", float(tv + tk) * D * es),
+        "similarity_gemm": ("tensor", sum(2.0 * (v - k) * k * D for v, k in zip(V, K))),
+        "members": ("hbm", 4.0 * tv + 4.0 * tv + 8.0 * tk),
+        "aggregate_compact": ("hbm", float(step.total + step.total_out) * D * es),
+        "proj_qkv": ("tensor", 2.0 * step.total_out * D * 3 * D),
+        "attn_post": ("tensor", sum(4.0 * n * n * D for n in step.out_lens_h)),
+    }
+
+
+def kernel_profile(step, run_host, q, peaks, n_steps=10):
+    """Device time of every kernel of the step while whole steps run back to back (CUDA profiling interface through
+    torch.profiler, outside any timed region), with its algorithmic work and the fraction of each peak it reaches."""
+    import torch
+    from torch.profiler import ProfilerActivity, profile
+    from paper_2511_12280_b200 import binding as B_
+    try:
+        # without launch overlap: otherwise a kernel's recorded time includes its wait for the drain of the one before
+        B_.d3tom_set_launch_overlap(False)
+        try:
+            for _ in range(2):
+                run_host()
+            torch.cuda.synchronize()
+            with profile(activities=[ProfilerActivity.CUDA]) as prof:
+                for _ in range(n_steps):
+                    run_host()
+                torch.cuda.synchronize()
+        finally:
+            B_.d3tom_set_launch_overlap(True)
+        evs = []
+        for e in prof.events():
+            if str(getattr(e, "device_type", "")).endswith("CUDA") and not e.name.lower().startswith(("memcpy", "memset")):
+                evs.append((e.time_range.start, e.name, float(e.time_range.elapsed_us())))
+        evs.sort()
+        seq = step_kernel_labels(step)
+        L = len(seq)
+        if L == 0 or len(evs) != L * n_steps:
+            return {"error": "expected %d kernels per step, the profiler saw %d in %d steps" % (L, len(evs), n_steps)}
+        times = {}
+        for i, (_, name, us) in enumerate(evs):
+            label, must = seq[i % L]
+            if must not in name:
+                return {"error": "kernel %d of a step is %s, expected %s" % (i % L, name[:60], label)}
+            times.setdefault(label, []).append(us)
+        work = kernel_work(step, q)
+        out = {}
+        per_step = 0.0
+        for label, _ in dict.fromkeys(seq):
+            ts = times[label]
+            us = float(np.median(ts))
+            calls = len(ts) // n_steps
+            per_step += us * calls
+            bound, amount = work[label]
+            rate = amount / (us * 1e-6)
+            entry = {"us": us, "launches_per_step": calls, "bound": bound}
+            if bound == "tensor":
+                tf = rate / 1e12
+                entry.update(gflop=amount / 1e9, tflops=tf, frac_nominal=tf / NOMINAL_PEAKS["bf16_tflops"],
+                             frac_measured_burst=tf / peaks["bf16_tflops"],
+                             frac_measured_sustained=tf / peaks["bf16_tflops_sustained"])
+            else:
+                gbs = rate / 1e9
+                entry.update(mbytes=amount / 1e6, gbs=gbs, frac_nominal=gbs / NOMINAL_PEAKS["hbm_gbs"],
+                             frac_measured_copy=gbs / peaks["hbm_gbs"])
+            out[label] = entry
+        out["sum_us_per_step"] = per_step
+        out["how"] = ("median device time over %d host-launched steps run back to back with the launch overlap "
+                      "(programmatic dependent launch) switched off, so that each kernel's time is its own; the timed "
+                      "step keeps the overlap, which hides most of every kernel's ramp-up and drain" % n_steps)
+        return out
+    except Exception as exc:                         # the profile is a report, never a reason to lose the bench line
+        return {"error": "%s: %s" % (type(exc).__name__, exc)}
+
+
+def block_timings(step, w, w_post0, q, dev, timed, reps):
     """The rest of a post-merge block (Algorithm 1, FFN_l; layer-cost equation of the FLOPs appendix): output
     projection and gated feed-forward network at the shortened length N_m, and the whole block at N_m and at the
     full length N, so that the measured saving of a post-merge layer can be set beside the FLOPs ratio.
@@ -256,80 +424,22 @@ def make_kv_cache_case(step, w, k, v, dev):
                                       cu_out_d, assign, mc, src)
 
 
-# ------------------------------------------------------------------------------------------ main
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", default="C2", choices=sorted(WORKLOAD_TEXT))
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-block", action="store_true", help="skip the timing of the rest of a post-merge block")
-    ap.add_argument("--tokens-per-step", type=int, default=1,
-                    help="schedule config: response tokens revealed per denoising step (2 gives T = 32 for 64 tokens)")
-    ap.add_argument("--reversed", action="store_true", help="schedule config: the high->low ablation of the schedule")
-    ap.add_argument("--deciders", default="all", choices=["all", "recent"],
-                    help="schedule config: every token revealed so far, or only those of the previous step")
-    ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
-    ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
-                    help="profiling aid: after one full step, run just this call --steps times and exit")
-    args = ap.parse_args()
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-
-    from paper_2511_12280_b200 import workload as wl
-    config = {"workload": WORKLOAD_TEXT[args.config], "requests_per_gpu": None, "aggregation": "mean",
-              "l2": "inputs larger than L2 (per-step working set > 126 MB)", "parallelism": "request-sharded replicas x%d" % world}
-
-    if args.impl == "reference":
-        if rank != 0:
-            return 0
-        w = wl.config(args.config)
-        config["requests_per_gpu"] = w.B
-        ref_kw = {}
-        if w.T:        # the schedule config is sampled at its middle step
-            from oracle import d3tom_oracle as orc
-            sm = w.T // 2
-            a_min = 2.0 * (1.0 - w.mean_keep_ratio) - 1.0
-            ref_kw = dict(decider_pos=w.step_deciders(sm),
-                          keep=[orc.keep_count(w.n_visual[0], 1.0 - orc.schedule_alpha(sm, w.T, a_min, 1.0))])
-            config["sampled_step"] = sm
-        times = []
-        desc, parts = "", {}
-        for i in range(args.warmup + args.steps):
-            sec, desc, parts = oracle_step_sample(w, **ref_kw)
-            if i >= args.warmup:
-                times.append(sec)
-        us = float(np.mean(times)) * 1e6
-        line = {"impl": "reference", "metric": "merge_layer_step_us", "value": us, "unit": "us", "n_gpus": args.gpus,
-                "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
-                "cpu_baseline": {"value": us, "unit": "us", "cores": blas_threads(), "kind": "oracle", "sample": desc},
-                "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-                "breakdown_s": parts}
-        print(json.dumps(line))
-        return 0
-
+# ------------------------------------------------------------------------------------------ one configuration on the GPU
+def measure_config(name, args, dev, local_rank, world, full):
+    """Times configuration ``name`` on this rank's GPU.  ``full`` adds the clock record, the per-kernel profile, the
+    K/V-cache merge, the rest of a post-merge block and the serial end-to-end figure (the chosen configuration);
+    without it only the step, its calls, the attention kernel alone and the overlapped end-to-end path are timed
+    (the other configurations of the `configs` object)."""
     import torch
     import torch.distributed as dist
     from paper_2511_12280_b200 import binding as B_
-    from paper_2511_12280_b200.pipeline import MergeLayerStep
-    from paper_2511_12280_b200 import replicas
-    from paper_2511_12280_b200 import trajectory
+    from paper_2511_12280_b200 import replicas, trajectory
+    from paper_2511_12280_b200 import workload as wl
+    from paper_2511_12280_b200.pipeline import HostFedStep, MergeLayerStep
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the merge-layer path has no CPU fallback")
-    B_.load()           # fails loudly if the CUDA library has not been built
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    w = wl.config(args.config)
-    config["requests_per_gpu"] = w.B
+    w = wl.config(name)
     total = int(w.cu_seqlens[-1])
+    res = {"requests_per_gpu": w.B, "total_tokens": total}
     # one problem per schedule step (a single one for the constant-ratio configs)
     plan = plan_unmerged = None
     if w.T:
@@ -341,23 +451,24 @@ def main():
                                                  merged=False, **kw_plan)
         dec_steps = [p.decider_pos for p in plan]
         keep_steps = [p.keep_count for p in plan]
-        config["schedule"] = {"T": T_steps, "alpha_min": a_min, "alpha_max": a_max, "tokens_per_step": args.tokens_per_step,
-                              "reversed": bool(args.reversed), "deciders": args.deciders,
-                              "keep_counts": [k[0] for k in keep_steps]}
+        res["schedule"] = {"T": T_steps, "alpha_min": a_min, "alpha_max": a_max, "tokens_per_step": args.tokens_per_step,
+                           "reversed": bool(args.reversed), "deciders": args.deciders,
+                           "keep_counts": [k[0] for k in keep_steps]}
     else:
         dec_steps = [w.decider_pos]
         keep_steps = [[B_.d3tom_keep_count(v, r) for v, r in zip(w.n_visual, w.keep_ratio)]]
     n_prob = len(dec_steps)
+    mid = n_prob // 2
     step = MergeLayerStep(w.H, w.dh, w.torch_dtype, total, w.B, max(sum(len(d) for d in dec) for dec in dec_steps),
                           max(w.n_visual), n_post=len(w.w_post), mode=B_.AGG_MEAN, device=local_rank)
     probs = [step.make_problem(w.n_visual, w.n_prompt, w.n_resp, dec, keep) for dec, keep in zip(dec_steps, keep_steps)]
-    step.use_problem(probs[n_prob // 2])
+    step.use_problem(probs[mid])
     q_hs = [w.q_for(dec).contiguous().pin_memory() for dec in dec_steps]
     k_h, v_h = w.k.contiguous().pin_memory(), w.v.contiguous().pin_memory()
     qs = [t.to(dev) for t in q_hs]
-    q_h, q = q_hs[n_prob // 2], qs[n_prob // 2]
+    q = qs[mid]
     k, v = k_h.to(dev), v_h.to(dev)
-    q_stage = torch.empty_like(q)               # where the end-to-end path lands the step's Q
+    q_stage = torch.empty_like(q)               # where the serial end-to-end path lands the step's Q
     w_post = [x.to(dev) for x in w.w_post]
     out_h = torch.empty(total, step.D, dtype=w.torch_dtype).pin_memory()
 
@@ -375,8 +486,16 @@ def main():
         e1.synchronize()
         return e0.elapsed_time(e1) / iters * 1e3   # us
 
-    def max_over_ranks(x):
-        return replicas.max_over_ranks(x, dev)
+    def timed_each(fn, iters):
+        """(mean over the whole region, per-iteration times): one event between consecutive iterations."""
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        ev[0].record()
+        for i in range(iters):
+            fn()
+            ev[i + 1].record()
+        ev[-1].synchronize()
+        each = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(iters)]
+        return ev[0].elapsed_time(ev[-1]) / iters * 1e3, each
 
     counter = {"i": 0, "launches": 0}
     # one CUDA graph per problem: a step is then one graph launch (the kernels and their order are unchanged)
@@ -386,8 +505,8 @@ def main():
         for i in range(n_prob):
             step.use_problem(probs[i])
             graphs.append(step.capture(qs[i], k, v, w_post))
-        step.use_problem(probs[n_prob // 2])
-    config["launch"] = "cuda graph replay, one per step" if graphs is not None else "host launches"
+        step.use_problem(probs[mid])
+    res["launch"] = "cuda graph replay, one per step" if graphs is not None else "host launches"
 
     def run():
         i = counter["i"] % n_prob
@@ -399,19 +518,24 @@ def main():
             return step.layer_out[-1] if step.n_post else step.hidden_out
         return step.run(qs[i], k, v, w_post)
 
+    def run_host_mid():
+        step.use_problem(probs[mid])
+        return step.run(qs[mid], k, v, w_post)
+
     if args.only is not None:
         run()
         calls = {
             "attn_importance": lambda: step.attn_importance(q, k, v),
             "select": lambda: step.select(),
             "merge": lambda: step.merge(),
-            "proj_qkv": lambda: step.ctx.d3tom_proj_qkv(step.hidden_out, w_post[0], step.total_out, step.D,
-                                                        step.q2, step.k2, step.v2),
-            "attn_varlen": lambda: step.ctx.d3tom_attn_varlen(step.q2, step.k2, step.v2, step.cu_out, step.nB,
-                                                              step.total_out, step.max_out, step.scale,
-                                                              step.layer_out[0]),
             "step": run,
         }
+        if step.n_post:
+            calls["proj_qkv"] = lambda: step.ctx.d3tom_proj_qkv(step.hidden_out, w_post[0], step.total_out, step.D,
+                                                                step.q2, step.k2, step.v2)
+            calls["attn_varlen"] = lambda: step.ctx.d3tom_attn_varlen(step.q2, step.k2, step.v2, step.cu_out, step.nB,
+                                                                      step.total_out, step.max_out, step.scale,
+                                                                      step.layer_out[0])
         if args.only in ("proj_out", "ffn"):          # the rest of a post-merge block at the shortened length
             m_ff = 3 * step.D
             t = wl.block_inputs(1000, 8, step.D, m_ff, w.dtype)
@@ -424,22 +548,26 @@ def main():
                                                       step.D, m_ff, act, y)
         torch.cuda.synchronize()
         us = timed(calls[args.only], args.steps)
-        print(json.dumps({"only": args.only, "us": us, "config": args.config}))
-        return 0
+        return {"only": args.only, "us": us, "config": name}
 
+    n_steps = args.steps if full else max(n_prob, min(args.steps, 40))
     # ---- device-resident timing of the whole step
     for _ in range(max(3, args.warmup)):
         run()
     sync_all()
-    with ClockSampler(local_rank) as clk:
-        clk.wait_started(run)          # keeps the GPU busy until the sampler delivers
+    clk_cm = ClockSampler(local_rank) if full else None
+    if clk_cm is not None:
+        clk_cm.__enter__()
+        clk_cm.wait_started(run)          # keeps the GPU busy until the sampler delivers
+    try:
         sync_all()
+        counter["i"] = 0
         counter["launches"] = 0
-        step_us = timed(run, args.steps)
-        launches_timed = counter["launches"]
+        step_us, each = timed_each(run, n_steps)
+        res["gpu_launches"] = counter["launches"]
+        res["steps_timed"] = n_steps
         sync_all()
         # ---- per-step series of the schedule config: one event pair per denoising step, median of 3 trajectories
-        per_step = None
         if w.T:
             series = []
             for _ in range(3):
@@ -453,12 +581,13 @@ def main():
             traj_u.run()
             sync_all()
             unmerged_us = float(np.median([timed(traj_u.run, 1) for _ in range(3)]))
-            traj_info = {"T": len(plan), "total_us": float(sum(per_step)), "unmerged_total_us": unmerged_us,
-                         "time_ratio": float(sum(per_step)) / unmerged_us,
-                         "flops_ratio": traj_m.flops(step.D, step.n_post) / traj_u.flops(step.D, step.n_post)}
+            res["per_step_us"] = per_step
+            res["trajectory"] = {"T": len(plan), "total_us": float(sum(per_step)), "unmerged_total_us": unmerged_us,
+                                 "time_ratio": float(sum(per_step)) / unmerged_us,
+                                 "flops_ratio": traj_m.flops(step.D, step.n_post) / traj_u.flops(step.D, step.n_post)}
             del traj_u
         # the breakdown below is taken at the middle problem
-        counter["i"] = n_prob // 2
+        counter["i"] = mid
         run()
         sync_all()
         # ---- per-call breakdown (each call timed back to back on warm instruction caches;
@@ -466,7 +595,6 @@ def main():
         reps = min(100, max(10, args.steps))
         # the dominant kernel alone (no importance side-work): the attention kernel at the merge-layer length; taken
         # first, before the long GEMM timings below pull the board into its power cap
-        sync_all()
         time.sleep(0.5)      # the burst peak it is compared with was measured on an idle board: let the power state settle
         attn_kernel_us = timed(lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
                                                                   step.max_seqlen, step.scale, step.attn_out), reps)
@@ -480,24 +608,36 @@ def main():
             br["attn_varlen"] = timed(lambda: step.ctx.d3tom_attn_varlen(step.q2, step.k2, step.v2, step.cu_out, step.nB,
                                                                         step.total_out, step.max_out, step.scale,
                                                                         step.layer_out[0]), reps)
-        # the same routing applied to the cached K/V prefix (Sec. 4.4): caches = K, V rows of [visual | prompt]
-        kv = make_kv_cache_case(step, w, k, v, dev)
-        br["merge_kv"] = timed(kv, reps)
-        # the rest of a post-merge block at N_m and at N (tensor-core path: bf16, widths in multiples of 128)
         block = None
-        if step.n_post and w.dtype == "bf16" and step.D % 128 == 0 and not args.no_block:
-            block = block_timings(step, w, w_post[0], q, k, v, dev, timed, max(5, reps // 4))
-            br["proj_out"] = block["Nm"]["proj_out"]
-            br["ffn"] = block["Nm"]["ffn"]
+        if full:
+            # the same routing applied to the cached K/V prefix (Sec. 4.4): caches = K, V rows of [visual | prompt]
+            kv = make_kv_cache_case(step, w, k, v, dev)
+            br["merge_kv"] = timed(kv, reps)
+            # the rest of a post-merge block at N_m and at N (tensor-core path: bf16, widths in multiples of 128)
+            if step.n_post and w.dtype == "bf16" and step.D % 128 == 0 and not args.no_block:
+                block = block_timings(step, w, w_post[0], q, dev, timed, max(5, reps // 4))
+                br["proj_out"] = block["Nm"]["proj_out"]
+                br["ffn"] = block["Nm"]["ffn"]
         sync_all()
-    clocks = clk.summary()
+    finally:
+        if clk_cm is not None:
+            clk_cm.__exit__(None, None, None)
+    if clk_cm is not None:
+        res["clocks"] = clk_cm.summary()
     assert step.ctx.device_status() == 0, "device status word reports a kernel-side problem"
+
+    peaks, peak_kind = load_peaks()
+    # ---- every kernel of the step inside running steps (outside the timed regions)
+    if full and w.dtype == "bf16":
+        for _ in range(3):
+            run_host_mid()
+        torch.cuda.synchronize()
+        res["kernels"] = kernel_profile(step, run_host_mid, q, peaks)
 
     # ---- end to end through the C ABI with host buffers: H2D of Q,K,V, the step, D2H of the result.
     #      HostFedStep overlaps the input copy of the next step and the result copy of the previous one with the
     #      running step (two input slots, three streams); the serial figure (copy, run, copy on one stream) is
     #      reported beside it.
-    from paper_2511_12280_b200.pipeline import HostFedStep
     e2e_bytes = {"h2d": 0, "d2h": 0, "n": 0}
     # (graphs only with a single problem: with one graph per schedule step and slot on top of the graphs above, replay
     #  was measured slower than host launches, 1.8 against 1.0 ms per step; the copies bound this path either way)
@@ -536,33 +676,36 @@ def main():
     e2e_bytes.update(h2d=0, d2h=0, n=0)
     e2e_us = timed_fed(max(n_prob, min(50, max(5, args.steps // 2))))
     sync_all()
-    for _ in range(3):
-        e2e_serial()
-    sync_all()
-    counter["i"] = 0
-    e2e_serial_us = timed(e2e_serial, max(n_prob, min(20, max(5, args.steps // 4))))
-    sync_all()
-    step.use_problem(probs[n_prob // 2])
+    e2e_serial_us = None
+    if full:
+        for _ in range(3):
+            e2e_serial()
+        sync_all()
+        counter["i"] = 0
+        e2e_serial_us = timed(e2e_serial, max(n_prob, min(20, max(5, args.steps // 4))))
+        sync_all()
+    step.use_problem(probs[mid])
 
-    step_us_max = max_over_ranks(step_us)
-    e2e_us_max = max_over_ranks(e2e_us)
+    step_us_max = replicas.max_over_ranks(step_us, dev)
+    e2e_us_max = replicas.max_over_ranks(e2e_us, dev)
 
     # ---- roofline of the dominant kernel (merge-layer attention): 4 N^2 D flops per request
-    peaks, peak_kind = load_peaks()
     attn_flops = sum(4.0 * n * n * step.D for n in step.seqlens_h)
     achieved = attn_flops / (attn_kernel_us * 1e-6) / 1e12
-    roofline = {"bound": "tensor", "kernel": "attn_tc_kernel (merge-layer attention, timed alone)",
-                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": ATTN_TRAFFIC_BYTES.get(args.config),
-                "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of one merge-layer launch with the "
-                                "importance spill (profiles/attn_tc_kernel_c2_merge_layer.md); algorithmic bytes "
-                                "%.1f MB" % (4 * step.total * step.D * q.element_size() / 1e6),
-                "peak_kind": peak_kind + " burst"}
+    res["roofline"] = {"bound": "tensor", "kernel": "attn_tc_kernel (merge-layer attention, timed alone)",
+                       "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                       "frac": achieved / peaks["bf16_tflops"], "traffic": ATTN_TRAFFIC_BYTES.get(name),
+                       "algorithmic_bytes": 4.0 * step.total * step.D * q.element_size(),
+                       "peak_kind": peak_kind + " burst",
+                       "frac_nominal": achieved / NOMINAL_PEAKS["bf16_tflops"],
+                       "frac_measured_sustained": achieved / peaks["bf16_tflops_sustained"],
+                       "us": attn_kernel_us}
     merge_bytes = (step.total + step.total_out) * step.D * q.element_size()
     sim_flops = sum(2.0 * (v_ - k_) * k_ * step.D for v_, k_ in zip(step.n_visual_h, step.keep_h))
     post_attn_flops = sum(4.0 * n * n * step.D for n in step.out_lens_h)
     derived = {
         "attn_importance_tflops": attn_flops / (br["attn_importance"] * 1e-6) / 1e12,
+        "attn_importance_frac_of_burst": attn_flops / (br["attn_importance"] * 1e-6) / 1e12 / peaks["bf16_tflops"],
         "merge_call_gbs": merge_bytes / (br["merge"] * 1e-6) / 1e9,
         "merge_call_frac_of_hbm_peak": merge_bytes / (br["merge"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
         "similarity_gflop": sim_flops / 1e9,
@@ -570,37 +713,129 @@ def main():
     if step.n_post:
         derived["attn_varlen_tflops"] = post_attn_flops / (br["attn_varlen"] * 1e-6) / 1e12
         derived["proj_qkv_tflops"] = 2.0 * step.total_out * step.D * 3 * step.D / (br["proj_qkv"] * 1e-6) / 1e12
-
-    line = {
-        "metric": "merge_layer_step_us", "value": step_us_max / world, "unit": "us", "n_gpus": world,
-        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": step_us_max / 1e3,
-        "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
-        "steps_per_s": world / (step_us_max * 1e-6),
-        "e2e": {"value": e2e_us_max / world, "unit": "us",
-                "h2d_bytes_per_step": int(e2e_bytes["h2d"] // max(1, e2e_bytes["n"])),
-                "d2h_bytes_per_step": int(e2e_bytes["d2h"] // max(1, e2e_bytes["n"])),
-                "how": "copies of neighbouring steps overlap the running step (two input slots, three streams)",
-                "serial_us": e2e_serial_us / world},
-        "gpu_launches": int(launches_timed),
-        "roofline": roofline, "breakdown_us": br, "derived": derived, "clocks": clocks,
-        "peaks": dict(peaks, kind=peak_kind),
-    }
-
+    res.update(step_us=step_us_max, step_us_this_rank=step_us, step_us_median=float(np.median(each)),
+               step_us_min=float(np.min(each)), breakdown_us=br, derived=derived, dtype=w.dtype,
+               e2e={"value": e2e_us_max / world, "unit": "us",
+                    "h2d_bytes_per_step": int(e2e_bytes["h2d"] // max(1, e2e_bytes["n"])),
+                    "d2h_bytes_per_step": int(e2e_bytes["d2h"] // max(1, e2e_bytes["n"])),
+                    "how": "copies of neighbouring steps overlap the running step (two input slots, three streams)"})
+    if e2e_serial_us is not None:
+        res["e2e"]["serial_us"] = e2e_serial_us / world
     if block is not None:
-        line["block"] = block
-    if per_step is not None:
-        line["per_step_us"] = per_step
-        line["trajectory_total_us"] = float(sum(per_step))
-        line["trajectory"] = traj_info
+        res["block"] = block
+    res["peaks"] = dict(peaks, kind=peak_kind)
+    res["_workload"] = w
+    res["_mid"] = (dec_steps[mid], keep_steps[mid], mid)
+    step.ctx.close()
+    return res
+
+
+# ------------------------------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="C2", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-block", action="store_true", help="skip the timing of the rest of a post-merge block")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--tokens-per-step", type=int, default=1,
+                    help="schedule config: response tokens revealed per denoising step (2 gives T = 32 for 64 tokens)")
+    ap.add_argument("--reversed", action="store_true", help="schedule config: the high->low ablation of the schedule")
+    ap.add_argument("--deciders", default="all", choices=["all", "recent"],
+                    help="schedule config: every token revealed so far, or only those of the previous step")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
+    ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
+                    help="profiling aid: after one full step, run just this call --steps times and exit")
+    args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        return spawn_ranks(args)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    config = {"workload": WORKLOAD_TEXT[args.config], "requests_per_gpu": None, "aggregation": "mean",
+              "l2": "inputs larger than L2 (per-step working set > 126 MB)",
+              "parallelism": "request-sharded replicas x%d" % world,
+              "unit_of_work": "one merge-layer step of one request batch of the workload; every GPU runs its own batch, "
+                              "value = slowest rank's time per step / number of GPUs"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        return reference_arm(args, config)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2511_12280_b200 import binding as B_
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the merge-layer path has no CPU fallback")
+    if local_rank >= torch.cuda.device_count():
+        raise SystemExit("rank %d has no GPU: %d visible" % (local_rank, torch.cuda.device_count()))
+    B_.load()           # fails loudly if the CUDA library has not been built
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    res = measure_config(args.config, args, dev, local_rank, world, full=True)
+    if args.only is not None:
+        print(json.dumps(res))
+        return 0
+    w = res.pop("_workload")
+    mid_dec, mid_keep, mid = res.pop("_mid")
+    config["requests_per_gpu"] = res.pop("requests_per_gpu")
+    config["launch"] = res.pop("launch")
+    if "schedule" in res:
+        config["schedule"] = res.pop("schedule")
+    step_us = res.pop("step_us")
+    line = {
+        "metric": "merge_layer_step_us", "value": step_us / world, "unit": "us", "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": step_us / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if res.pop("dtype") == "bf16" else "f32", "data": "synthetic", "config": config,
+        "steps_per_s": world / (step_us * 1e-6),
+        "step_us_median": res.pop("step_us_median"), "step_us_min": res.pop("step_us_min"),
+        "e2e": res.pop("e2e"), "gpu_launches": int(res.pop("gpu_launches")),
+        "roofline": res.pop("roofline"), "breakdown_us": res.pop("breakdown_us"), "derived": res.pop("derived"),
+        "clocks": res.pop("clocks"), "peaks": res.pop("peaks"),
+    }
+    res.pop("step_us_this_rank", None); res.pop("steps_timed", None); res.pop("total_tokens", None)
+    if "per_step_us" in res:
+        line["per_step_us"] = res["per_step_us"]
+        line["trajectory_total_us"] = float(sum(res.pop("per_step_us")))
+    line.update(res)                       # kernels, block, trajectory
+
+    # ---- the other configurations, briefly (one GPU; the chosen configuration is the one the metric is quoted on)
+    if world == 1 and not args.no_configs:
+        others = {}
+        for name in ("C1", "C3", "C4"):
+            if name == args.config:
+                continue
+            r = measure_config(name, args, dev, local_rank, world, full=False)
+            o = {"workload": WORKLOAD_TEXT[name], "step_us": r["step_us"], "step_us_median": r["step_us_median"],
+                 "step_us_min": r["step_us_min"], "steps_timed": r["steps_timed"],
+                 "attn_kernel_us": r["roofline"]["us"], "attn_tflops": r["roofline"]["achieved"],
+                 "attn_frac": r["roofline"]["frac"], "attn_frac_nominal": r["roofline"]["frac_nominal"],
+                 "e2e_us": r["e2e"]["value"], "h2d_bytes_per_step": r["e2e"]["h2d_bytes_per_step"],
+                 "d2h_bytes_per_step": r["e2e"]["d2h_bytes_per_step"], "breakdown_us": r["breakdown_us"]}
+            if "trajectory" in r:
+                o["trajectory"] = r["trajectory"]
+            others[name] = o
+        line["configs"] = others
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         kw = {}
         if w.T:
-            kw = dict(decider_pos=dec_steps[n_prob // 2], keep=keep_steps[n_prob // 2])
-            config["cpu_baseline_step"] = n_prob // 2
-        sec, desc, parts = oracle_step_sample(w, **kw)
+            kw = dict(decider_pos=mid_dec, keep=mid_keep)
+            config["cpu_baseline_step"] = mid
+        sec, parts = oracle_step(w, oracle_inputs(w, kw.get("decider_pos")), **kw)
         line["cpu_baseline"] = {"value": sec * 1e6, "unit": "us", "cores": blas_threads(), "kind": "oracle",
-                                "sample": desc, "breakdown_s": parts}
+                                "sample": ORACLE_SAMPLE_TEXT, "steps_timed": 1, "extrapolated": False,
+                                "breakdown_s": parts}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

@@ -91,6 +91,15 @@ int64_t d3tom_workspace_bytes(const d3tom_ctx* ctx);
  * kernels that serve fp32 (slow; lets the two code paths be compared on the GPU). */
 int d3tom_set_reference_kernels(d3tom_ctx* ctx, int on);
 
+/* Profiling aid, process-wide.  By default every kernel of the library is launched so
+ * that its thread blocks may become resident while the kernel before it in the stream
+ * drains (programmatic dependent launch; each kernel still waits for its predecessor's
+ * results before it reads them).  A profiler then attributes that waiting to the later
+ * kernel.  With on == 0 kernels start only after their predecessor has finished, so
+ * per-kernel device times are separable (and a step is a little slower); results are
+ * the same either way.  Not thread-safe against concurrent launches. */
+int d3tom_set_launch_overlap(int on);
+
 /* Sec. 3.2.1, "Rank(S_j) <= (1-alpha)|V|": number of kept tokens for keep
  * ratio r = 1-alpha.  Host arithmetic: clamp(floor(r*n_visual + 1e-9), 1, n_visual). */
 int d3tom_keep_count(int n_visual, double keep_ratio);

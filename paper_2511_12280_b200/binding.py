@@ -45,6 +45,7 @@ _SIGNATURES = {
     "d3tom_device_status": (_I, [_P, C.POINTER(_I)]),
     "d3tom_workspace_bytes": (C.c_int64, [_P]),
     "d3tom_set_reference_kernels": (_I, [_P, _I]),
+    "d3tom_set_launch_overlap": (_I, [_I]),
     "d3tom_keep_count": (_I, [_I, C.c_double]),
     "d3tom_schedule_alpha": (_I, [_I, _I, C.c_double, C.c_double, _I, C.POINTER(C.c_double)]),
     "d3tom_attn_importance": (_I, [_P, _I, _P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _F, _P, _P, _P, _P]),
@@ -111,6 +112,12 @@ def _dt(t: torch.Tensor) -> int:
 # ------------------------------------------------------------------ host helpers
 def d3tom_keep_count(n_visual: int, keep_ratio: float) -> int:
     return load().d3tom_keep_count(int(n_visual), float(keep_ratio))
+
+
+def d3tom_set_launch_overlap(on: bool):
+    """Profiling aid: with on = False kernels start only after their predecessor has finished (separable per-kernel
+    device times); the default lets a kernel's blocks become resident while its predecessor drains."""
+    _check(load().d3tom_set_launch_overlap(int(on)), "d3tom_set_launch_overlap")
 
 
 def d3tom_schedule_alpha(step: int, T: int, a_min: float, a_max: float, reversed_: bool = False) -> float:

@@ -5,6 +5,8 @@
 
 #include "common.cuh"
 
+int g_d3tom_launch_overlap = 1;
+
 namespace {
 
 struct DeviceGuard {
@@ -131,6 +133,11 @@ int64_t d3tom_workspace_bytes(const d3tom_ctx* ctx) { return ctx ? ctx->bytes : 
 int d3tom_set_reference_kernels(d3tom_ctx* ctx, int on) {
   if (ctx == nullptr) return D3TOM_ERR_INVALID_ARG;
   ctx->reference_kernels = on ? 1 : 0;
+  return D3TOM_OK;
+}
+
+int d3tom_set_launch_overlap(int on) {
+  g_d3tom_launch_overlap = on ? 1 : 0;
   return D3TOM_OK;
 }
 

@@ -65,12 +65,15 @@ __device__ __forceinline__ void grid_dependency_enter() {
   grid_dependency_release();
 }
 
+// Process-wide switch behind d3tom_set_launch_overlap (1 = overlap, the default).
+extern int g_d3tom_launch_overlap;
+
 template <typename... Params, typename... Args>
 inline cudaError_t launch_serialized(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
                                      Args&&... args) {
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[0].val.programmaticStreamSerializationAllowed = g_d3tom_launch_overlap ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
   cfg.attrs = attr; cfg.numAttrs = 1;
