@@ -84,6 +84,18 @@ int d3tom_last_cuda_error(const d3tom_ctx* ctx);
 /* Copies the device-side status word to *status_out (host).  Synchronises the
  * device; call it after the stream work of interest has been waited for. */
 int d3tom_device_status(d3tom_ctx* ctx, int* status_out);
+/* Sets the device-side status word back to 0 (synchronises the device first). */
+int d3tom_reset_device_status(d3tom_ctx* ctx);
+/* Self-test of the bounded waits.  Every wait inside the library's kernels (on a
+ * barrier that a copy, the tensor pipe or another warp completes) gives up after a
+ * time limit, records D3TOM_ERR_TIMEOUT in the status word and lets the kernel release
+ * what it holds and return, so that a wait that cannot end costs that limit and not a
+ * hung GPU.  This call enqueues a one-block kernel that waits, with the same routine
+ * and a limit of `limit_ns` (1 .. 10^9), on a barrier that nothing completes: after the
+ * stream has been waited for, d3tom_device_status reports D3TOM_ERR_TIMEOUT and the
+ * context is usable as before (clear the word with d3tom_reset_device_status).
+ * The kernel issues no copy and no tensor-core instruction and faults nothing. */
+int d3tom_selftest_wait_timeout(d3tom_ctx* ctx, int64_t limit_ns, d3tom_stream stream);
 /* Bytes of scratch the context holds (host query). */
 int64_t d3tom_workspace_bytes(const d3tom_ctx* ctx);
 

@@ -43,6 +43,8 @@ _SIGNATURES = {
     "d3tom_status_string": (C.c_char_p, [_I]),
     "d3tom_last_cuda_error": (_I, [_P]),
     "d3tom_device_status": (_I, [_P, C.POINTER(_I)]),
+    "d3tom_reset_device_status": (_I, [_P]),
+    "d3tom_selftest_wait_timeout": (_I, [_P, C.c_int64, _P]),
     "d3tom_workspace_bytes": (C.c_int64, [_P]),
     "d3tom_set_reference_kernels": (_I, [_P, _I]),
     "d3tom_set_launch_overlap": (_I, [_I]),
@@ -171,6 +173,13 @@ class Context:
         out = C.c_int()
         _check(load().d3tom_device_status(self._h, C.byref(out)), "d3tom_device_status")
         return out.value
+
+    def reset_device_status(self):
+        _check(load().d3tom_reset_device_status(self._h), "d3tom_reset_device_status")
+
+    def selftest_wait_timeout(self, limit_ns: int, stream=None):
+        """Enqueues the one-block kernel whose wait cannot end; afterwards device_status() is ERR_TIMEOUT."""
+        _check(load().d3tom_selftest_wait_timeout(self._h, int(limit_ns), _stream(stream)), "d3tom_selftest_wait_timeout")
 
     # -------------------------------------------------------------- the four calls (+ projection)
     def d3tom_attn_importance(self, q, k, v, cu_seqlens, n_visual, decider_pos, cu_deciders, B, total_tokens,

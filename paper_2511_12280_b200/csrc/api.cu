@@ -128,6 +128,21 @@ int d3tom_device_status(d3tom_ctx* ctx, int* status_out) {
   return D3TOM_OK;
 }
 
+int d3tom_reset_device_status(d3tom_ctx* ctx) {
+  if (ctx == nullptr) return D3TOM_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  D3TOM_CUDA_TRY(ctx, cudaDeviceSynchronize());
+  D3TOM_CUDA_TRY(ctx, cudaMemset(ctx->dev_status, 0, sizeof(int)));
+  return D3TOM_OK;
+}
+
+int d3tom_selftest_wait_timeout(d3tom_ctx* ctx, int64_t limit_ns, d3tom_stream stream) {
+  if (ctx == nullptr || limit_ns <= 0 || limit_ns > 1000000000ll) return D3TOM_ERR_INVALID_ARG;   // at most one second
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return D3TOM_ERR_CUDA;
+  return launch_wait_timeout_selftest(ctx, (long long)limit_ns, static_cast<cudaStream_t>(stream));
+}
+
 int64_t d3tom_workspace_bytes(const d3tom_ctx* ctx) { return ctx ? ctx->bytes : 0; }
 
 int d3tom_set_reference_kernels(d3tom_ctx* ctx, int on) {

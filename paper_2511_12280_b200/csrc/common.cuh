@@ -180,6 +180,8 @@ int launch_merge_finish(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);    
 int launch_merge_aggregate(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);   // aggregate, compact (lists already built)
 int launch_merge_aggregate_stream(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s);   // the same as a bulk-copy pipeline
 
+int launch_wait_timeout_selftest(d3tom_ctx* ctx, long long limit_ns, cudaStream_t s);   // a wait that cannot end
+
 int launch_proj_simt(d3tom_ctx* ctx, d3tom_dtype dt, const void* x, const void* w, int total, int D,
                      void* q, void* k, void* v, cudaStream_t s);
 int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int D,

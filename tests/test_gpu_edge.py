@@ -217,3 +217,32 @@ def test_results_are_reproducible_run_to_run():
         for a, b in zip(outs[0], o):
             assert torch.equal(a, b)
     step.ctx.close()
+
+
+def test_a_wait_that_cannot_end_reports_timeout_and_leaves_the_context_usable():
+    # the library's wait routine on a barrier that nothing completes, with a 3 ms limit: the kernel returns, the status
+    # word says so, and after clearing it the same context computes a correct step
+    import time
+    w = small(post=0)
+    step = pu.make_step(w, sim_debug=False)
+    dev = step.dev
+    q, k, v = w.q_for().to(dev), w.k.to(dev), w.v.to(dev)
+    assert step.ctx.device_status() == 0
+    t0 = time.time()
+    step.ctx.selftest_wait_timeout(3_000_000)
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 1.0                       # it gave up after its limit: nothing hung
+    assert step.ctx.device_status() == B_.ERR_TIMEOUT
+    step.ctx.reset_device_status()
+    assert step.ctx.device_status() == 0
+    with pytest.raises(B_.D3tomError) as e:             # the limit is bounded on the host: at most one second
+        step.ctx.selftest_wait_timeout(5_000_000_000)
+    assert e.value.status == B_.ERR_INVALID_ARG
+    step.run(q, k, v)
+    torch.cuda.synchronize()
+    assert step.ctx.device_status() == 0
+    scale = 1.0 / np.sqrt(w.dh)
+    want = orc.round_storage(orc.attention(pu.f64(w.q_for()), pu.f64(w.k), pu.f64(w.v), w.cu_seqlens, scale), w.dtype)
+    pu.assert_close(pu.f64(step.attn_out[:step.total]), want, w.dtype, "attention output after a timed-out wait")
+    pu.assert_guard_rows_untouched(step)
+    step.ctx.close()
