@@ -122,7 +122,7 @@ constexpr int kMaxPrefixBatch = 64;     // ragged batches up to this many reques
 template <int BN, int EPI, int MT = 1>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
-  static_assert(MT == 1 || (BN == 256 && EPI != kEpiSim), "the 256-row tile serves the dense layers at 256 columns");
+  static_assert(MT == 1 || (BN >= 224 && BN % 32 == 0 && EPI != kEpiSim), "the 256-row tile serves the dense layers at 224 or 256 columns");
   using S = GemmSmem<BN, MT>;
   constexpr int kStages = S::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -340,7 +340,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           // 32 divides D, so a 32-column piece lies in one of q, k, v even when the tile straddles two of them
           const int gcol = tc.n0 + c, which = gcol / p.out_cols;
           __nv_bfloat16* dst = p.out[which] + (size_t)grow * p.out_cols + (gcol - which * p.out_cols) - c;
-          if (grow < p.out_rows) {
+          if (grow < p.out_rows && which < 3) {      // (a tile width that does not divide 3 D: the last tile hangs over)
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
               uint32_t w[4];
@@ -359,7 +359,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (int c = 0; c < BN; c += 32) {
           float r[32];
           load32(c, r);
-          if (grow < p.out_rows) {
+          if (grow < p.out_rows && tc.n0 + c < p.ld_out) {
             const size_t off = (size_t)grow * p.ld_out + tc.n0 + c;
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
@@ -487,18 +487,26 @@ void plan_tail_split(const d3tom_ctx* ctx, GemmParams& p) {
 }
 
 // Which tile shape finishes a dense layer sooner, from measured main-loop cycles per 64 of K (projection timings at
-// 128 .. 4288 rows).  128 x 256 tiles: 850 per full round over the SMs (48 KB of operands per k-block: what the SMs
+// 128 .. 7600 rows).  128 x 256 tiles: 850 per full round over the SMs (48 KB of operands per k-block: what the SMs
 // together can pull out of L2), and 150 + 3.9 r for a last round of r tiles, which runs faster per tile because
 // fewer SMs share L2.  256 x 256 tiles: 1450 per full round (64 KB per k-block in three 64 KB stages: bound by the
-// load latency of one SM, so a round of few tiles is no cheaper), 900 + 3.5 r for the last round.  The larger tile
-// wins when it saves a round of the smaller one.
-bool prefer_two_m_tiles(const d3tom_ctx* ctx, int rows, int n_tiles_256) {
+// load latency of one SM, so a round of few tiles is no cheaper), 900 + 3.5 r for the last round; 256 x 224 tiles
+// cost 0.89 of that per round and sometimes need a round less, or fill the last one better (1216 rows x 12288
+// columns: 275 tiles in two rounds, 93 us against 99 us for the 240 tiles of 256 x 256).
+// Returns the width of the 256-row tile to use (256 or 224), or 0 for 128-row tiles.
+int two_m_tile_width(const d3tom_ctx* ctx, int rows, int ncols, bool allow_224) {
   const int sms = ctx->sm_count;
-  const long long t1 = (long long)ceil_div(rows, kBM) * n_tiles_256, t2 = (long long)ceil_div(rows, 2 * kBM) * n_tiles_256;
-  const double r1 = (double)(t1 % sms), r2 = (double)(t2 % sms);
+  const long long t1 = (long long)ceil_div(rows, kBM) * ceil_div(ncols, 256);
+  const double r1 = (double)(t1 % sms);
   const double cost1 = 850.0 * (double)(t1 / sms) + (r1 > 0 ? 150.0 + 3.9 * r1 : 0.0);
-  const double cost2 = 1450.0 * (double)(t2 / sms) + (r2 > 0 ? 900.0 + 3.5 * r2 : 0.0);
-  return cost2 < 0.97 * cost1;
+  auto cost2 = [&](int width, double scale) {
+    const long long t2 = (long long)ceil_div(rows, 2 * kBM) * ceil_div(ncols, width);
+    const double r2 = (double)(t2 % sms);
+    return scale * (1450.0 * (double)(t2 / sms) + (r2 > 0 ? 900.0 + 3.5 * r2 : 0.0));
+  };
+  const double c256 = ncols % 256 == 0 ? cost2(256, 1.0) : 1e30, c224 = allow_224 ? cost2(224, 0.89) : 1e30;
+  if (c224 < 0.97 * c256 && c224 < 0.97 * cost1) return 224;
+  return c256 < 0.97 * cost1 ? 256 : 0;
 }
 
 template <int BN, int EPI, int MT = 1>
@@ -557,11 +565,12 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  if ((3 * D) % 256 == 0 && prefer_two_m_tiles(ctx, total, 3 * D / 256)) {
+  if (const int w2 = two_m_tile_width(ctx, total, 3 * D, D % 32 == 0)) {
     r = make_tmap_bf16_2d(&ta, x, (uint64_t)total, (uint64_t)D, (uint64_t)D, 2 * kBM);
-    if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 256);
+    if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, (uint32_t)w2);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-    p.m_tiles = ceil_div(total, 2 * kBM); p.n_tiles = 3 * D / 256;
+    p.m_tiles = ceil_div(total, 2 * kBM); p.n_tiles = ceil_div(3 * D, w2);
+    if (w2 == 224) return launch_gemm<224, kEpiProj, 2>(ctx, ta, tb, p, s);
     return launch_gemm<256, kEpiProj, 2>(ctx, ta, tb, p, s);
   }
   r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, (uint32_t)bn);
@@ -593,11 +602,12 @@ int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* r
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  if (N % 256 == 0 && prefer_two_m_tiles(ctx, rows, N / 256)) {
+  if (const int w2 = two_m_tile_width(ctx, rows, N, true)) {
     r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)K, (uint64_t)K, 2 * kBM);
-    if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, 256);
+    if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)w2);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-    p.m_tiles = ceil_div(rows, 2 * kBM); p.n_tiles = N / 256;
+    p.m_tiles = ceil_div(rows, 2 * kBM); p.n_tiles = ceil_div(N, w2);
+    if (w2 == 224) return launch_gemm<224, kEpiLinear, 2>(ctx, ta, tb, p, s);
     return launch_gemm<256, kEpiLinear, 2>(ctx, ta, tb, p, s);
   }
   r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)bn);
@@ -621,7 +631,7 @@ int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int 
   p.dev_status = ctx->dev_status;
   p.m_tiles = ceil_div(rows, kBM); p.n_tiles = m / 128; p.batch = 1; p.k_splits = 1;
   {
-    if (prefer_two_m_tiles(ctx, rows, m / 128)) {
+    if (two_m_tile_width(ctx, rows, 2 * m, false) == 256) {
       r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)D, (uint64_t)D, 2 * kBM);
       if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
       p.m_tiles = ceil_div(rows, 2 * kBM);

@@ -62,6 +62,10 @@ def test_linear_and_ffn_bf16_shapes_that_take_256_row_tiles():
     run_linear(1500, 64, 12288, "bf16", residual=True, seed=5)
     run_linear(1500, 128, 12288, "bf16", residual=False, seed=6)
     run_ffn(1500, 128, 6144, "bf16", seed=7)
+    # 1216 rows x 12288 columns: 256 x 224 tiles (275 of them fill two rounds over 148 SMs better than 240 tiles of
+    # 256 x 256); 224 does not divide 12288, so the last column tile hangs over the edge of the matrix
+    run_linear(1216, 64, 12288, "bf16", residual=True, seed=8)
+    run_linear(1216, 128, 12288, "bf16", residual=False, seed=9)
 
 
 def test_linear_fp32_odd_sizes():
