@@ -33,7 +33,9 @@
  *    D3TOM_ERR_WORKSPACE; nothing is reallocated.  Two calls on the same
  *    context must not overlap on the GPU (use one context per stream).
  *  - Every function returns a status: D3TOM_OK (0) or a negative error.  No
- *    exceptions, no abort, nothing printed.  Argument errors are detected on
+ *    exceptions, no abort, nothing printed (unless the environment variable
+ *    D3TOM_LOG is set to something other than 0: then d3tom_create and the four
+ *    calls of the path write one line per call, sizes and status, to stderr).  Argument errors are detected on
  *    the host before anything is launched.  Problems only the device can see
  *    (a bounded wait that ran out) are recorded in a status word read by
  *    d3tom_device_status.

@@ -1,6 +1,9 @@
 // C ABI of the D3ToM merge-layer library: context, host helpers, argument
 // validation and dispatch to the kernels.  See include/d3tom.h for the contract.
 #include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <new>
 
 #include "common.cuh"
@@ -8,6 +11,23 @@
 int g_d3tom_launch_overlap = 1;
 
 namespace {
+
+// D3TOM_LOG=1 in the environment: one line per call on stderr (sizes and the status returned).  Read once.
+bool log_enabled() {
+  static const int on = [] { const char* e = getenv("D3TOM_LOG"); return (e != nullptr && e[0] != '\0' && e[0] != '0') ? 1 : 0; }();
+  return on != 0;
+}
+int logged(int status, const char* fmt, ...) {
+  if (log_enabled()) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    fprintf(stderr, "[d3tom] %s -> %d (%s)\n", buf, status, d3tom_status_string(status));
+  }
+  return status;
+}
 
 struct DeviceGuard {
   int prev = -1;
@@ -48,7 +68,17 @@ int check_head_dim(const d3tom_ctx* ctx, d3tom_dtype dt) {
 
 extern "C" {
 
+static int create_impl(d3tom_ctx** out, int device, const d3tom_limits* lim);
+
 int d3tom_create(d3tom_ctx** out, int device, const d3tom_limits* lim) {
+  const int st = create_impl(out, device, lim);
+  if (lim == nullptr) return logged(st, "d3tom_create device %d", device);
+  return logged(st, "d3tom_create device %d: tokens %d batch %d heads %d x %d deciders %d visual %d, scratch %lld bytes", device,
+                lim->max_total_tokens, lim->max_batch, lim->heads, lim->head_dim, lim->max_deciders,
+                lim->max_visual_per_request, (long long)((st == D3TOM_OK && out && *out) ? (*out)->bytes : 0));
+}
+
+static int create_impl(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (out == nullptr || lim == nullptr) return D3TOM_ERR_INVALID_ARG;
   *out = nullptr;
   if (lim->max_total_tokens <= 0 || lim->max_batch <= 0 || lim->heads <= 0 || lim->head_dim <= 0 ||
@@ -225,21 +255,35 @@ int d3tom_attn_importance(d3tom_ctx* ctx, d3tom_dtype dt, const void* q, const v
                           const int32_t* cu_deciders, int B, int total_tokens, int max_seqlen, int max_visual,
                           int n_deciders_total, float softmax_scale, void* attn_out, float* importance,
                           const int32_t* cu_vis, d3tom_stream stream) {
-  return attn_common(ctx, dt, q, k, v, cu_seqlens, n_visual, decider_pos, cu_deciders, B, total_tokens, max_seqlen,
-                     max_visual, n_deciders_total, softmax_scale, attn_out, importance, cu_vis, true,
-                     static_cast<cudaStream_t>(stream));
+  return logged(attn_common(ctx, dt, q, k, v, cu_seqlens, n_visual, decider_pos, cu_deciders, B, total_tokens, max_seqlen,
+                            max_visual, n_deciders_total, softmax_scale, attn_out, importance, cu_vis, true,
+                            static_cast<cudaStream_t>(stream)),
+                "d3tom_attn_importance dt %d B %d tokens %d max_seqlen %d max_visual %d deciders %d", (int)dt, B, total_tokens,
+                max_seqlen, max_visual, n_deciders_total);
 }
 
 int d3tom_attn_varlen(d3tom_ctx* ctx, d3tom_dtype dt, const void* q, const void* k, const void* v,
                       const int32_t* cu_seqlens, int B, int total_tokens, int max_seqlen, float softmax_scale,
                       void* out, d3tom_stream stream) {
-  return attn_common(ctx, dt, q, k, v, cu_seqlens, nullptr, nullptr, nullptr, B, total_tokens, max_seqlen, 0, 0,
-                     softmax_scale, out, nullptr, nullptr, false, static_cast<cudaStream_t>(stream));
+  return logged(attn_common(ctx, dt, q, k, v, cu_seqlens, nullptr, nullptr, nullptr, B, total_tokens, max_seqlen, 0, 0,
+                            softmax_scale, out, nullptr, nullptr, false, static_cast<cudaStream_t>(stream)),
+                "d3tom_attn_varlen dt %d B %d tokens %d max_seqlen %d", (int)dt, B, total_tokens, max_seqlen);
 }
+
+static int select_impl(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis, const int32_t* keep_count,
+                       const int32_t* cu_kept, int B, int max_visual, int32_t* kept_idx, uint8_t* keep_mask,
+                       d3tom_stream stream);
 
 int d3tom_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis, const int32_t* keep_count,
                  const int32_t* cu_kept, int B, int max_visual, int32_t* kept_idx, uint8_t* keep_mask,
                  d3tom_stream stream) {
+  return logged(select_impl(ctx, importance, cu_vis, keep_count, cu_kept, B, max_visual, kept_idx, keep_mask, stream),
+                "d3tom_select B %d max_visual %d", B, max_visual);
+}
+
+static int select_impl(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis, const int32_t* keep_count,
+                       const int32_t* cu_kept, int B, int max_visual, int32_t* kept_idx, uint8_t* keep_mask,
+                       d3tom_stream stream) {
   if (ctx == nullptr || importance == nullptr || cu_vis == nullptr || keep_count == nullptr || cu_kept == nullptr ||
       kept_idx == nullptr || keep_mask == nullptr || B <= 0 || max_visual < 0)
     return D3TOM_ERR_INVALID_ARG;
@@ -299,9 +343,11 @@ int d3tom_merge(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* hidd
                 int B, int D, int total_tokens, int total_out, int max_visual, int max_kept, void* hidden_out,
                 const int32_t* cu_seqlens_out, int32_t* assign, int32_t* member_count, int32_t* src_of_dst,
                 float* sim_debug, d3tom_stream stream) {
-  return merge_common(ctx, dt, mode, hidden, nullptr, cu_seqlens, n_visual, cu_vis, kept_idx, cu_kept, B, D,
-                      total_tokens, total_out, max_visual, max_kept, hidden_out, nullptr, cu_seqlens_out, assign,
-                      member_count, src_of_dst, sim_debug, static_cast<cudaStream_t>(stream));
+  return logged(merge_common(ctx, dt, mode, hidden, nullptr, cu_seqlens, n_visual, cu_vis, kept_idx, cu_kept, B, D,
+                             total_tokens, total_out, max_visual, max_kept, hidden_out, nullptr, cu_seqlens_out, assign,
+                             member_count, src_of_dst, sim_debug, static_cast<cudaStream_t>(stream)),
+                "d3tom_merge dt %d mode %d B %d D %d tokens %d -> %d max_visual %d max_kept %d", (int)dt, (int)mode, B, D,
+                total_tokens, total_out, max_visual, max_kept);
 }
 
 int d3tom_merge_kv(d3tom_ctx* ctx, d3tom_dtype dt, d3tom_agg mode, const void* k_cache, const void* v_cache,

@@ -94,3 +94,22 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert not re.search(r"(import\s+oracle|from\s+oracle|oracle[./]d3tom|oracle/)", src), os.path.join(dirpath, f)
+
+
+def test_log_line_per_call_when_the_environment_asks_for_it():
+    # D3TOM_LOG=1: one line per call on stderr with sizes and status; silent otherwise.  Without a GPU
+    # d3tom_create fails on the host, which is enough to see both behaviours.
+    import subprocess
+    import sys
+    code = ("from paper_2511_12280_b200 import binding as B\n"
+            "try:\n    B.Context(128, 1, 2, 64, 1, 64).close()\nexcept B.D3tomError:\n    pass\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    for val, expect in (("1", True), ("0", False), (None, False)):
+        env = dict(os.environ)
+        env.pop("D3TOM_LOG", None)
+        if val is not None:
+            env["D3TOM_LOG"] = val
+        r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
+        has = "[d3tom] d3tom_create device 0: tokens 128 batch 1 heads 2 x 64" in r.stderr
+        assert has == expect, (val, r.stderr)
