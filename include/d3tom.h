@@ -168,7 +168,11 @@ int d3tom_attn_importance(d3tom_ctx* ctx, d3tom_dtype dt,
  * packed tokens, fits exactly).
  *
  * heads, head_dim replace the context's limits; every other argument is as in
- * d3tom_attn_importance, and the results are the same bit for bit.  The work
+ * d3tom_attn_importance.  The results are those of d3tom_attn_importance to
+ * rounding: bit for bit where that call runs the same whole-item kernel, within
+ * the tolerances of the parity tests where it balances a single request's work
+ * items over the SMs (that path keeps partial tiles in context scratch, which
+ * this entry point does not have).  The work
  * runs on the CURRENT device, which must be the one `stream` and the buffers
  * belong to.  device_status_out (device, nullable) receives the kernels'
  * status word at the end of the call (0, or D3TOM_ERR_TIMEOUT if a bounded

@@ -53,6 +53,7 @@ void free_all(d3tom_ctx* c) {
   cudaFree(c->inv_norm_kept); cudaFree(c->kept_rows); cudaFree(c->best); cudaFree(c->member_off);
   cudaFree(c->member_cursor); cudaFree(c->member_list); cudaFree(c->heavy_slots); cudaFree(c->n_heavy); cudaFree(c->row_desc); cudaFree(c->agg_counter);
   cudaFree(c->gemm_split_ws); cudaFree(c->gemm_split_counters); cudaFree(c->dev_status);
+  cudaFree(c->attn_part_ws); cudaFree(c->attn_part_flags);
 }
 
 bool dtype_ok(d3tom_dtype dt) { return dt == D3TOM_BF16 || dt == D3TOM_FP32; }
@@ -121,6 +122,9 @@ static int create_impl(d3tom_ctx** out, int device, const d3tom_limits* lim) {
   if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_ws, (size_t)2 * c->sm_count * 128 * 256);
   if (st == D3TOM_OK) st = alloc(c, &c->gemm_split_counters, (size_t)2 * c->sm_count);
   if (st == D3TOM_OK && cudaMemset(c->gemm_split_counters, 0, 2 * c->sm_count * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
+  if (st == D3TOM_OK) st = alloc(c, &c->attn_part_ws, (size_t)c->sm_count * 2 * (128 + 2) * 128);
+  if (st == D3TOM_OK) st = alloc(c, &c->attn_part_flags, (size_t)c->sm_count * 8);
+  if (st == D3TOM_OK && cudaMemset(c->attn_part_flags, 0, (size_t)c->sm_count * 8 * sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st == D3TOM_OK) st = alloc(c, &c->dev_status, 1);
   if (st == D3TOM_OK && cudaMemset(c->dev_status, 0, sizeof(int)) != cudaSuccess) st = D3TOM_ERR_CUDA;
   if (st != D3TOM_OK) { free_all(c); delete c; return st; }
@@ -240,8 +244,12 @@ static int attn_common(d3tom_ctx* ctx, d3tom_dtype dt, const void* q, const void
   a.score_scratch = ctx->score_scratch; a.lse_scratch = ctx->lse_scratch;
   a.max_deciders = ctx->lim.max_deciders > 0 ? ctx->lim.max_deciders : 1; a.vis_stride = ctx->vis_stride;
   a.dev_status = ctx->dev_status;
-  if (dt == D3TOM_BF16 && !ctx->reference_kernels) st = launch_attn_tc(ctx, a, stream);
-  else st = launch_attn_simt(ctx, dt, a, stream);
+  if (dt == D3TOM_BF16 && !ctx->reference_kernels) {
+    st = launch_attn_sk(ctx, a, stream);                       // one request whose items do not fill whole rounds of SMs
+    if (st == D3TOM_ERR_UNSUPPORTED) st = launch_attn_tc(ctx, a, stream);
+  } else {
+    st = launch_attn_simt(ctx, dt, a, stream);
+  }
   if (st != D3TOM_OK) return st;
   if (with_importance) {
     a.cu_deciders = cu_deciders;

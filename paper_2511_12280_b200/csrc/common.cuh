@@ -32,6 +32,8 @@ struct d3tom_ctx {
   int4* row_desc;               // [max_total_tokens] per output row: {source row, members or -1, list offset, request start}
   float* gemm_split_ws;         // [2 * sm_count][256][128] fp32 partial similarity tiles (K slices of a tile)
   int* gemm_split_counters;     // [2 * sm_count] slices done per tile; zero between launches
+  float* attn_part_ws;          // [sm_count][2][128 + 2][128] fp32: O tile and (m, l) of an attention item's later key tiles
+  int* attn_part_flags;         // [sm_count][2][4] one word per (CTA, query tile, warp); zero between launches
   int* dev_status;              // device status word
   int vis_stride;               // row stride of score_scratch (floats)
 };
@@ -159,6 +161,7 @@ struct AttnArgs {
 
 int launch_attn_simt(d3tom_ctx* ctx, d3tom_dtype dt, const AttnArgs& a, cudaStream_t s);
 int launch_attn_tc(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s);
+int launch_attn_sk(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s);      // one request, work balanced over the SMs
 int launch_importance_finish(d3tom_ctx* ctx, const AttnArgs& a, int max_visual, float* importance,
                              const int32_t* cu_vis, cudaStream_t s);
 int launch_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis, const int32_t* keep_count,
