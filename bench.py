@@ -50,7 +50,7 @@ WORKLOAD_TEXT = {
 }
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the committed ncu
 # capture; null for configurations not captured, and null whenever attn_tc.cu has changed since the capture
-ATTN_TRAFFIC_BYTES = {"C2": 164.8e6}
+ATTN_TRAFFIC_BYTES = {"C2": 194.7e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 REFERENCE_BUDGET_S = 240.0          # the CPU arm stops adding steps once they would not fit this

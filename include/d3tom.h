@@ -86,7 +86,9 @@ int d3tom_last_cuda_error(const d3tom_ctx* ctx);
 /* Copies the device-side status word to *status_out (host).  Synchronises the
  * device; call it after the stream work of interest has been waited for. */
 int d3tom_device_status(d3tom_ctx* ctx, int* status_out);
-/* Sets the device-side status word back to 0 (synchronises the device first). */
+/* Sets the device-side status word back to 0 (synchronises the device first) and
+ * returns the counters and flags that kernels leave at zero between launches to that
+ * state: call it after D3TOM_ERR_TIMEOUT was reported, before the context is used again. */
 int d3tom_reset_device_status(d3tom_ctx* ctx);
 /* Self-test of the bounded waits.  Every wait inside the library's kernels (on a
  * barrier that a copy, the tensor pipe or another warp completes) gives up after a

@@ -167,6 +167,12 @@ int d3tom_reset_device_status(d3tom_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   D3TOM_CUDA_TRY(ctx, cudaDeviceSynchronize());
   D3TOM_CUDA_TRY(ctx, cudaMemset(ctx->dev_status, 0, sizeof(int)));
+  // a kernel that gave up may have left its self-cleaning counters and flags behind: back to their resting state
+  const size_t n_ctr = (size_t)ctx->lim.max_batch * (((size_t)ctx->lim.max_visual_per_request + 255) / 256);
+  D3TOM_CUDA_TRY(ctx, cudaMemset(ctx->imp_counters, 0, n_ctr * sizeof(int)));
+  D3TOM_CUDA_TRY(ctx, cudaMemset(ctx->agg_counter, 0, 2 * sizeof(int)));
+  D3TOM_CUDA_TRY(ctx, cudaMemset(ctx->gemm_split_counters, 0, (size_t)2 * ctx->sm_count * sizeof(int)));
+  D3TOM_CUDA_TRY(ctx, cudaMemset(ctx->attn_part_flags, 0, (size_t)ctx->sm_count * 8 * sizeof(int)));
   return D3TOM_OK;
 }
 

@@ -71,19 +71,27 @@ __device__ __forceinline__ bool flag_wait(const int* flag, int want, volatile in
 }
 
 // The CTA's walk over its share [pos, hi) of the step line: one segment = (item, key tiles [j0, j1)).
+// The line holds, head by head, the n_kv steps of each of the head's nqb items and then `pad` empty positions:
+// the head's last item carries the response rows, and when those spill their scores for the importance map its
+// steps cost about a quarter more; the empty positions charge that to the share that gets them.
 struct Walk {
-  int pos, hi, n_kv, nqb, n;
+  int pos, hi, n_kv, nqb, n, pad;
   int t, j0, j1, h, q0, n_qt;
   __device__ __forceinline__ bool next() {
-    if (pos >= hi) return false;
-    t = pos / n_kv;
-    j0 = pos - t * n_kv;
-    j1 = min(n_kv, j0 + (hi - pos));
-    h = t / nqb;
-    q0 = (t - h * nqb) * 2 * kTile;
-    n_qt = (n - q0 > kTile) ? 2 : 1;
-    pos += j1 - j0;
-    return true;
+    const int head_len = nqb * n_kv + pad;
+    while (pos < hi) {
+      h = pos / head_len;
+      const int r = pos - h * head_len, qb = r / n_kv;
+      if (qb >= nqb) { pos += min(head_len - r, hi - pos); continue; }      // empty positions: nothing to do
+      j0 = r - qb * n_kv;
+      j1 = min(n_kv, j0 + (hi - pos));
+      t = h * nqb + qb;
+      q0 = qb * 2 * kTile;
+      n_qt = (n - q0 > kTile) ? 2 : 1;
+      pos += j1 - j0;
+      return true;
+    }
+    return false;
   }
 };
 
@@ -99,15 +107,19 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   constexpr int kSlotFloats = 2 * (128 + 2) * kTile;     // per CTA: two tiles of [128 columns][128 rows] + (m, l) per row
   grid_dependency_enter();
   const int lo = a.cu_seqlens[0], n = a.cu_seqlens[1] - lo;
+  // deciders are response rows: rows below the visual count cannot be any, and their segments skip the look-up
+  const int n_vis = a.decider_pos != nullptr ? a.n_visual[0] : 0;
+  const int dec_lo = a.decider_pos != nullptr ? a.cu_deciders[0] : 0, dec_hi = a.decider_pos != nullptr ? a.cu_deciders[1] : 0;
   const int nqb = (n + 2 * kTile - 1) / (2 * kTile), n_kv = (n + kTile - 1) / kTile;
-  const int items = a.H * nqb;
-  const int G = min((int)gridDim.x, items);              // a share must be at least one item long
+  const int pad = a.decider_pos != nullptr ? (n_kv + 2) / 4 : 0;
+  const long long W = (long long)a.H * (nqb * n_kv + pad);
+  // a share must be at least one item (and its empty positions) long, so that an item is cut at most once
+  const int G = (int)min((long long)gridDim.x, W / (n_kv + pad));
   const int cta = (int)blockIdx.x;
   if (cta >= G || n <= 0) return;                        // uniform; nothing allocated yet
-  const long long W = (long long)items * n_kv;
   Walk walk0;
   walk0.pos = (int)((long long)cta * W / G); walk0.hi = (int)((long long)(cta + 1) * W / G);
-  walk0.n_kv = n_kv; walk0.nqb = nqb; walk0.n = n;
+  walk0.n_kv = n_kv; walk0.nqb = nqb; walk0.n = n; walk0.pad = pad;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -267,10 +279,9 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const bool last_tile = i == w.n_qt - 1;                  // its warps release the K/V stages
       const int q_row = w.q0 + i * kTile + row;
       const bool valid_row = q_row < n;
-      int dec_slot = -1, n_vis = 0;
-      if (a.decider_pos != nullptr && valid_row) {
-        n_vis = a.n_visual[0];
-        int l = a.cu_deciders[0], r = a.cu_deciders[1];
+      int dec_slot = -1;
+      if (a.decider_pos != nullptr && valid_row && q_row >= n_vis) {
+        int l = dec_lo, r = dec_hi;
         while (l < r) {
           const int mid = (l + r) >> 1, pos = a.decider_pos[mid];
           if (pos == q_row) { dec_slot = mid; break; }
@@ -352,20 +363,6 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           exp_chunk(0, m_used, pk[0], l_tile);
           exp_chunk(1, m_used, pk[1], l_tile);
         }
-        if (score_row != nullptr && j * kTile < n_vis) {
-          const int key0 = j * kTile;
-#pragma unroll
-          for (int e = 0; e < kTile; e += 4) {
-            if (key0 + e + 3 < n_vis) {
-              *reinterpret_cast<float4*>(score_row + key0 + e) =
-                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
-                              __uint_as_float(sr[e + 3]));
-            } else {
-#pragma unroll
-              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
-            }
-          }
-        }
         tmem_st16(t_s, pk[0]);
         tmem_st16(t_s + 16, pk[1]);
         exp_chunk(2, m_used, pk[0], l_tile);
@@ -385,6 +382,23 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&p_hi[i]);
+        // Decider rows: the raw scores over the visual keys go out AFTER P has been announced: the stores (one row per
+        // lane, 512 bytes each, uncoalesced) then run while the tensor pipe works on this tile instead of delaying it
+        // (the score registers stay live until the next key tile's load).
+        if (score_row != nullptr && j * kTile < n_vis) {
+          const int key0 = j * kTile;
+#pragma unroll
+          for (int e = 0; e < kTile; e += 4) {
+            if (key0 + e + 3 < n_vis) {
+              *reinterpret_cast<float4*>(score_row + key0 + e) =
+                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
+                              __uint_as_float(sr[e + 3]));
+            } else {
+#pragma unroll
+              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
+            }
+          }
+        }
       }
       // ---- end of the segment
       if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&o_final[i], seg_i & 1, abort_flag, a.dev_status));
@@ -489,12 +503,12 @@ int launch_attn_sk(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   const int items = a.H * ceil_div(a.max_seqlen, 2 * kTile), sms = ctx->sm_count;
   if (items <= sms) return D3TOM_ERR_UNSUPPORTED;
   // Whole items cost ceil(items / SMs) rounds.  The balanced walk pays a partial tile per CTA and an epilogue per
-  // segment, and its fixed shares cannot follow SMs that run a little slower than others: measured, it wins where a
-  // second round would be mostly idle (160 items on 148 SMs at 1216 rows: 37.2 against 43.4 us) and loses on long
-  // sequences (544 items at 4288 rows, 3.68 rounds: 285 against 272 us).  Taken for up to two rounds, when more than
-  // a twentieth of them would be idle.
+  // segment, so it is taken where more than a twentieth of those rounds would be idle.  Measured in one process,
+  // alternating (32 heads x 128, us, balanced / whole items): 1216 rows (1.08 rounds) 37.8 / 43.6, 1600 (1.51)
+  // 57.7 / 59.1, 2176 (1.95) 81.8 / 72.3, 2500 (2.16) 105.7 / 116.5, 3500 (3.03) 185 / 211, 4288 (3.68) 270 / 283,
+  // 6000 (5.19) 533 / 569, 8192 (6.92) 941 / 1026 (noisy under the power cap).
   const int rounds = ceil_div(items, sms);
-  if (rounds > 2 || (long long)(rounds * sms - items) * 20 <= (long long)rounds * sms) return D3TOM_ERR_UNSUPPORTED;
+  if ((long long)(rounds * sms - items) * 20 <= (long long)rounds * sms) return D3TOM_ERR_UNSUPPORTED;
   if (a.dh == 128) return launch<128>(ctx, a, s);
   if (a.dh == 64) return launch<64>(ctx, a, s);
   return D3TOM_ERR_UNSUPPORTED;

@@ -224,9 +224,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const uint32_t t_s = tmem + lane_addr + col_s(i);
       const uint32_t t_o = tmem + lane_addr + col_o(i);
       // is this row a decider of the request?
+      // (deciders are response rows: a row below the visual count cannot be one and skips the look-up)
       int dec_slot = -1, n_vis = 0;
-      if (a.decider_pos != nullptr && valid_row) {
-        n_vis = a.n_visual[b];
+      if (a.decider_pos != nullptr) n_vis = a.n_visual[b];
+      if (a.decider_pos != nullptr && valid_row && q_row >= n_vis) {
         int l = a.cu_deciders[b], r = a.cu_deciders[b + 1];
         while (l < r) {
           const int mid = (l + r) >> 1, pos = a.decider_pos[mid];
@@ -316,20 +317,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           exp_chunk(0, m_used, pk[0], l_tile);
           exp_chunk(1, m_used, pk[1], l_tile);
         }
-        if (score_row != nullptr && j * kTile < n_vis) {    // decider row: raw scores over the visual keys
-          const int key0 = j * kTile;
-#pragma unroll
-          for (int e = 0; e < kTile; e += 4) {
-            if (key0 + e + 3 < n_vis) {
-              *reinterpret_cast<float4*>(score_row + key0 + e) =
-                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
-                              __uint_as_float(sr[e + 3]));
-            } else {
-#pragma unroll
-              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
-            }
-          }
-        }
         // ---- the bf16 P tile goes into the first 64 columns of the S tile; the tensor pipe is told after each half
         tmem_st16(t_s, pk[0]);                             // keys 32*ch .. +31 -> P columns 16*ch .. +15
         tmem_st16(t_s + 16, pk[1]);
@@ -348,6 +335,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&p_hi[i]);
+        // Decider rows: the raw scores over the visual keys go out AFTER P has been announced: the stores (one row per
+        // lane, 512 bytes each, uncoalesced) then run while the tensor pipe works on this tile instead of delaying it
+        // (the score registers stay live until the next key tile's load).
+        if (score_row != nullptr && j * kTile < n_vis) {
+          const int key0 = j * kTile;
+#pragma unroll
+          for (int e = 0; e < kTile; e += 4) {
+            if (key0 + e + 3 < n_vis) {
+              *reinterpret_cast<float4*>(score_row + key0 + e) =
+                  make_float4(__uint_as_float(sr[e]), __uint_as_float(sr[e + 1]), __uint_as_float(sr[e + 2]),
+                              __uint_as_float(sr[e + 3]));
+            } else {
+#pragma unroll
+              for (int t = 0; t < 4; ++t) if (key0 + e + t < n_vis) score_row[key0 + e + t] = __uint_as_float(sr[e + t]);
+            }
+          }
+        }
       }
       // ---- epilogue: O / l -> bf16 -> global
       if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&o_final[i], 0, abort_flag, a.dev_status));
