@@ -95,7 +95,9 @@ struct Walk {
   }
 };
 
-template <int DH>
+// kImp: the launch also feeds the importance map (decider rows look themselves up and store their scores); the
+// plain instance carries none of that code, which keeps its softmax loop at the registers and schedule it had.
+template <int DH, bool kImp>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, AttnArgs a, float* __restrict__ part_ws,
@@ -108,10 +110,10 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   grid_dependency_enter();
   const int lo = a.cu_seqlens[0], n = a.cu_seqlens[1] - lo;
   // deciders are response rows: rows below the visual count cannot be any, and their segments skip the look-up
-  const int n_vis = a.decider_pos != nullptr ? a.n_visual[0] : 0;
-  const int dec_lo = a.decider_pos != nullptr ? a.cu_deciders[0] : 0, dec_hi = a.decider_pos != nullptr ? a.cu_deciders[1] : 0;
+  const int n_vis = (kImp && a.decider_pos != nullptr) ? a.n_visual[0] : 0;
+  const int dec_lo = (kImp && a.decider_pos != nullptr) ? a.cu_deciders[0] : 0, dec_hi = (kImp && a.decider_pos != nullptr) ? a.cu_deciders[1] : 0;
   const int nqb = (n + 2 * kTile - 1) / (2 * kTile), n_kv = (n + kTile - 1) / kTile;
-  const int pad = a.decider_pos != nullptr ? (n_kv + 2) / 4 : 0;
+  const int pad = (kImp && a.decider_pos != nullptr) ? (n_kv + 2) / 4 : 0;
   const long long W = (long long)a.H * (nqb * n_kv + pad);
   // a share must be at least one item (and its empty positions) long, so that an item is cut at most once
   const int G = (int)min((long long)gridDim.x, W / (n_kv + pad));
@@ -280,7 +282,7 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const int q_row = w.q0 + i * kTile + row;
       const bool valid_row = q_row < n;
       int dec_slot = -1;
-      if (a.decider_pos != nullptr && valid_row && q_row >= n_vis) {
+      if ((kImp && a.decider_pos != nullptr) && valid_row && q_row >= n_vis) {
         int l = dec_lo, r = dec_hi;
         while (l < r) {
           const int mid = (l + r) >> 1, pos = a.decider_pos[mid];
@@ -385,7 +387,7 @@ attn_sk_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // Decider rows: the raw scores over the visual keys go out AFTER P has been announced: the stores (one row per
         // lane, 512 bytes each, uncoalesced) then run while the tensor pipe works on this tile instead of delaying it
         // (the score registers stay live until the next key tile's load).
-        if (score_row != nullptr && j * kTile < n_vis) {
+        if (kImp && score_row != nullptr && j * kTile < n_vis) {
           const int key0 = j * kTile;
 #pragma unroll
           for (int e = 0; e < kTile; e += 4) {
@@ -487,8 +489,9 @@ int launch(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   if (r == 0) r = make_tmap_bf16_2d(&tk, a.k, rows, cols, cols, kTile);
   if (r == 0) r = make_tmap_bf16_2d(&tv, a.v, rows, cols, cols, kTile);
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_sk_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SkSmem<DH>::kBytes));
-  D3TOM_CUDA_TRY(ctx, launch_serialized(attn_sk_kernel<DH>, ctx->sm_count, kAttnThreads, SkSmem<DH>::kBytes, s, tq, tk, tv, a,
+  auto kernel = a.decider_pos != nullptr ? attn_sk_kernel<DH, true> : attn_sk_kernel<DH, false>;
+  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SkSmem<DH>::kBytes));
+  D3TOM_CUDA_TRY(ctx, launch_serialized(kernel, ctx->sm_count, kAttnThreads, SkSmem<DH>::kBytes, s, tq, tk, tv, a,
                                         ctx->attn_part_ws, ctx->attn_part_flags));
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;

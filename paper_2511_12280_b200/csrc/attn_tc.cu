@@ -60,7 +60,9 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 
-template <int DH>
+// kImp: the launch also feeds the importance map (decider rows look themselves up and store their scores); the
+// plain instance carries none of that code, which keeps its softmax loop at the registers and schedule it had.
+template <int DH, bool kImp>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, AttnArgs a) {
@@ -226,8 +228,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       // is this row a decider of the request?
       // (deciders are response rows: a row below the visual count cannot be one and skips the look-up)
       int dec_slot = -1, n_vis = 0;
-      if (a.decider_pos != nullptr) n_vis = a.n_visual[b];
-      if (a.decider_pos != nullptr && valid_row && q_row >= n_vis) {
+      if ((kImp && a.decider_pos != nullptr)) n_vis = a.n_visual[b];
+      if ((kImp && a.decider_pos != nullptr) && valid_row && q_row >= n_vis) {
         int l = a.cu_deciders[b], r = a.cu_deciders[b + 1];
         while (l < r) {
           const int mid = (l + r) >> 1, pos = a.decider_pos[mid];
@@ -338,7 +340,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // Decider rows: the raw scores over the visual keys go out AFTER P has been announced: the stores (one row per
         // lane, 512 bytes each, uncoalesced) then run while the tensor pipe works on this tile instead of delaying it
         // (the score registers stay live until the next key tile's load).
-        if (score_row != nullptr && j * kTile < n_vis) {
+        if (kImp && score_row != nullptr && j * kTile < n_vis) {
           const int key0 = j * kTile;
 #pragma unroll
           for (int e = 0; e < kTile; e += 4) {
@@ -393,8 +395,8 @@ int launch(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   if (r == 0) r = make_tmap_bf16_2d(&tk, a.k, rows, cols, cols, kTile);
   if (r == 0) r = make_tmap_bf16_2d(&tv, a.v, rows, cols, cols, kTile);
   if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
-  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           AttnSmem<DH>::kBytes));
+  auto kernel = a.decider_pos != nullptr ? attn_tc_kernel<DH, true> : attn_tc_kernel<DH, false>;
+  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<DH>::kBytes));
   AttnArgs k = a;
   k.nqb = ceil_div(a.max_seqlen, 2 * kTile);
   const int items = a.H * k.nqb, sms = ctx->sm_count > 0 ? ctx->sm_count : 1;
@@ -405,7 +407,7 @@ int launch(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
     else if (items > sms && rest > 0 && 2 * rest <= sms) k.split_from = items - rest;   // incomplete last wave
   }
   const int grid = a.B * (items + (items - k.split_from));
-  D3TOM_CUDA_TRY(ctx, launch_serialized(attn_tc_kernel<DH>, grid, kAttnThreads, AttnSmem<DH>::kBytes, s, tq, tk, tv, k));
+  D3TOM_CUDA_TRY(ctx, launch_serialized(kernel, grid, kAttnThreads, AttnSmem<DH>::kBytes, s, tq, tk, tv, k));
   D3TOM_LAUNCH_CHECK(ctx);
   return D3TOM_OK;
 }
