@@ -73,6 +73,29 @@ def test_single_request_balanced_walk_over_the_sms():
     pu.check_step(w)
 
 
+def test_balanced_walk_gives_the_same_bits_on_every_run():
+    # the halves of a cut item meet through global memory and a flag; the order of the two terms is fixed, so
+    # repeated launches on the same inputs (with other launches in between, which shifts the timing between CTAs)
+    # must agree bit for bit, for the rows and for the importance map
+    w = small(H=40, dh=128, reqs=[dict(V=900, P=33, O=70, n_dec=64, r=0.5)], post=0)
+    step = pu.make_step(w, sim_debug=False)
+    dev = step.dev
+    q, k, v = w.q_for().to(dev), w.k.to(dev), w.v.to(dev)
+    first = None
+    for it in range(25):
+        step.attn_out.fill_(float("nan")); step.importance.fill_(float("nan"))
+        step.attn_importance(q, k, v)
+        if it % 3 == 0:
+            step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, 1, step.total, step.max_seqlen, step.scale, step.hidden_out)
+        torch.cuda.synchronize()
+        got = (step.attn_out[:step.total].clone(), step.importance[:step.total_vis].clone())
+        if first is None:
+            first = got
+        assert torch.equal(got[0], first[0]) and torch.equal(got[1], first[1]), "run %d differs" % it
+    assert step.ctx.device_status() == 0
+    step.ctx.close()
+
+
 def test_kept_set_larger_than_the_shared_memory_counters():
     # more than 12288 kept tokens in one request: the member counters live in global memory, the bitmap of a
     # sorting warp spans 13000 positions, and select stages 13000 keys
