@@ -169,6 +169,11 @@ def test_keep_count_values():
     assert orc.keep_count(1000, 1 - 0.9) == 100     # 99.99999999999997 in binary
     assert orc.keep_count(256, 0.25) == 64
     assert orc.keep_count(4096, 0.25) == 1024
+    # the number of integer ranks 1..|V| that satisfy Rank <= x is floor(x), not the nearest integer
+    assert orc.keep_count(1026, 0.10) == 102        # 102.6
+    assert orc.keep_count(15, 0.5) == 7             # 7.5
+    assert orc.keep_count(7, 0.5) == 3              # 3.5
+    assert orc.keep_count(2048, 0.4999) == 1023     # 1023.8
     assert orc.keep_count(10, 0.0) == 1             # clamp below
     assert orc.keep_count(10, 1.0) == 10 and orc.keep_count(10, 1.5) == 10
 
