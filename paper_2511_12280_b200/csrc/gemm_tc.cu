@@ -29,7 +29,8 @@ constexpr int kBM = 128, kBK = 64;
 constexpr int kGemmThreads = 224;      // warps: 0 A loads, 1 MMA, 2..5 epilogue, 6 B loads
 
 enum { kEpiProj = 0, kEpiSim = 1, kEpiLinear = 2, kEpiGateUp = 3 };
-constexpr int kMaxKSplits = 4;        // K slices per similarity tile at most
+constexpr int kMaxKSplits = 4;        // K slices per tile at most when the last slice to arrive adds them all
+constexpr int kCoopSlices = 16;       // K slices per similarity tile at most when every slice adds its own share of the columns (8 or 16)
 
 struct GemmParams {
   int num_k_blocks;           // K / 64
@@ -38,6 +39,7 @@ struct GemmParams {
   int full_tiles;             // the first tiles of the walk are whole work units (0: every tile is cut)
   float* split_ws;            // [(tiles - full_tiles) * k_splits][BN][128] fp32 partial tiles (column-major: coalesced per warp)
   int* split_counters;        // [tiles] parts done; zero between launches
+  int coop;                   // similarity, few tiles: 8 or 16 slices per tile, all resident; each reduces BN / k_splits columns
   // projection
   __nv_bfloat16* out[3];      // q, k, v
   int out_rows;               // total tokens
@@ -273,6 +275,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // counter, left at zero again) adds the parts in the order of the K slices and runs the epilogue on
       // the sums: same values whichever unit comes last.
       const bool split = un.nsp > 1;
+      const bool coop = EPI == kEpiSim && p.coop != 0;
       const int ws_tile = t - p.full_tiles;                     // cut tiles are numbered from zero in the workspace
       bool last = true;
       if (split) {
@@ -292,9 +295,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (et == 0) s_prev = atomicAdd(p.split_counters + ws_tile, 1);
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        last = s_prev == un.nsp - 1;
-        if (last) {
-          if (et == 0) p.split_counters[ws_tile] = 0;
+        if (!coop) {
+          last = s_prev == un.nsp - 1;
+          if (last) {
+            if (et == 0) p.split_counters[ws_tile] = 0;
+            __threadfence();
+          }
+        } else {
+          // every slice of the tile is a CTA of its own and all of them are resident: wait (bounded) until all have
+          // written, then each adds up its own share of the columns
+          if (et == 0) {
+            const volatile int* ctr = p.split_counters + ws_tile;
+            const uint64_t t0 = ptx::globaltimer_ns();
+            uint32_t polls = 0;
+            s_prev = 1;
+            while (*ctr < un.nsp) {
+              if ((++polls & 0xffu) == 0u && (*abort_flag || ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs)) {
+                *abort_flag = 1;
+                atomicExch(p.dev_status, -5);
+                s_prev = 0;
+                break;
+              }
+            }
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (s_prev == 0) break;
           __threadfence();
         }
       }
@@ -328,6 +353,60 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
       };
       if (!last) { ++lt; continue; }
+      if (EPI == kEpiSim && coop) {
+        // this slice's share of the tile's columns, eight at a time: the sums over all slices (ascending slice
+        // order), then the arg-max over those columns; the 64-bit maximum over slices and tiles is order-independent
+        const int nsp = un.nsp;                                  // 8 or 16
+        const int cw = BN / nsp;
+        const int cb = sp * cw;
+        const int m = m_base + row;
+        const int g = tc.v0 + m;
+        const bool active = m < tc.Vb && p.assign[g] < 0;
+        const float inm = active ? p.inv_norm[g] : 0.f;
+        float best_sim = -INFINITY;
+        int best_slot = 0;
+        float* dbg = (p.sim_debug != nullptr && active) ? p.sim_debug + (size_t)g * p.max_kept + tc.n0 : nullptr;
+#pragma unroll 1
+        for (int c8 = cb; c8 < cb + cw; c8 += 8) {
+          float dot[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) dot[i] = 0.f;
+#pragma unroll 1
+          for (int q0 = 0; q0 < nsp; q0 += 8) {                  // eight slices' loads in flight at a time
+            float part[8][8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float* src = p.split_ws + ((size_t)(ws_tile * nsp + q0 + q) * BN + c8) * kBM + row;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) part[q][i] = __ldcg(src + (size_t)i * kBM);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q) dot[i] += part[q][i];
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int sidx = tc.n0 + c8 + i;
+            if (active && sidx < tc.kb) {
+              const float sim = (dot[i] * inm) * ink_s[c8 + i] + 0.0f;
+              if (sim > best_sim) { best_sim = sim; best_slot = sidx; }
+              if (dbg != nullptr) dbg[c8 + i] = sim;
+            }
+          }
+        }
+        if (active && tc.n0 + cb < tc.kb) {
+          const unsigned long long mine =
+              ((unsigned long long)ordered_key(best_sim) << 32) | (0xffffffffu - (unsigned)best_slot);
+          atomicMax(p.best + g, mine);
+        }
+        // the counter goes on to twice the slices as they finish reading; the last one leaves it at zero
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (et == 0 && atomicAdd(p.split_counters + ws_tile, 1) == 2 * nsp - 1) p.split_counters[ws_tile] = 0;
+        ++lt;
+        continue;
+      }
       // (a 256-row tile: the same epilogue once per 128-row half, each half in its own accumulator)
 #pragma unroll 1
       for (int mh = 0; mh < MT; ++mh, t_row += S::kAccStride, m_base += kBM) {
@@ -664,6 +743,15 @@ int launch_sim_tc(d3tom_ctx* ctx, const MergeArgs& a, cudaStream_t s) {
     if (splits > kMaxKSplits) splits = kMaxKSplits;
     if (splits > p.num_k_blocks) splits = p.num_k_blocks;
     if (splits < 2 || tiles * splits > 2LL * ctx->sm_count) splits = 1;
+    // very few tiles (a small kept set, one short request): eight or sixteen slices per tile, each a CTA of its
+    // own, and every slice adds up its share of the tile's columns itself instead of the last one adding all
+    for (int c = kCoopSlices; c >= 8; c /= 2) {
+      if (tiles * c <= ctx->sm_count && p.num_k_blocks >= 2 * c) {
+        splits = c;
+        p.coop = 1;
+        break;
+      }
+    }
     p.k_splits = splits;
     p.full_tiles = 0;                                   // every tile is cut (or none: one slice)
     p.split_ws = ctx->gemm_split_ws; p.split_counters = ctx->gemm_split_counters;

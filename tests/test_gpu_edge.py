@@ -104,6 +104,21 @@ def test_kept_set_larger_than_the_shared_memory_counters():
     pu.check_step(w, full_attention=False, n_sample_rows=6)
 
 
+@pytest.mark.parametrize("reqs", [
+    [dict(V=900, P=9, O=12, n_dec=4, r=0.1)],       # 8 tiles of 128 kept columns: sixteen K slices each
+    [dict(V=1500, P=5, O=8, n_dec=3, r=0.07)],      # 12 tiles of 128: eight slices each
+    [dict(V=1000, P=7, O=9, n_dec=2, r=0.2)],       # 8 tiles of 256: sixteen slices each
+    [dict(V=1000, P=7, O=9, n_dec=5, r=0.3)],       # 8 x 2 tiles of 256, the second 44 columns wide: eight slices
+    [dict(V=500, P=3, O=6, n_dec=2, r=0.12), dict(V=300, P=8, O=4, n_dec=4, r=0.33)],   # two requests, 4 + 3 tiles
+], ids=["128x16", "128x8", "256x16", "256x8", "batch"])
+def test_few_similarity_tiles_are_cut_along_k_and_every_slice_reduces_its_columns(reqs):
+    # a handful of (pruned rows x kept columns) tiles and a wide hidden vector: each tile's K range goes to 8 or 16
+    # CTAs, which wait for one another and then add up a share of the columns each
+    w = small(H=16, dh=128, reqs=reqs, post=0)
+    pu.check_step(w, full_attention=False, n_sample_rows=24)
+    pu.check_step(w, mode=B_.AGG_SUM, full_attention=False, n_sample_rows=24)
+
+
 def test_text_only_request_inside_a_batch():
     # a request without visual tokens between two ordinary ones: nothing to select or merge there, its rows are
     # copied, its attention runs as usual
