@@ -266,10 +266,10 @@ def step_kernel_labels(step):
     seq = [("attn_merge_layer", "attn_"), ("importance_finish", "importance_finish"), ("select", "select"),
            ("prepare_rows", "prepare_rows")]
     if step.total_out < step.total:
-        seq.append(("similarity_gemm", "gemm_tc"))
+        seq.append(("similarity_gemm", "gemm_"))
     seq += [("members", "members"), ("aggregate_compact", "aggregate")]
     for _ in range(step.n_post):
-        seq += [("proj_qkv", "gemm_tc"), ("attn_post", "attn_")]
+        seq += [("proj_qkv", "gemm_"), ("attn_post", "attn_")]       # gemm_tc_kernel, or gemm_pair_kernel for long layers
     return seq
 
 

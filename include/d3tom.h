@@ -116,6 +116,14 @@ int d3tom_set_reference_kernels(d3tom_ctx* ctx, int on);
  * the same either way.  Not thread-safe against concurrent launches. */
 int d3tom_set_launch_overlap(int on);
 
+/* Tile shape of the dense layers (d3tom_proj_qkv, d3tom_linear, d3tom_ffn; Sec. 3.2.1 "Q = H W_Q", Algorithm 1
+ * FFN_l): -1 (default) lets the library choose per shape (pairs from about two thousand rows on), 0 keeps single-CTA
+ * tiles, 256 forces tiles of 256 x 256 computed by a pair of CTAs (cta_group::2) wherever the number of output columns
+ * is a multiple of 256.  Results do not depend on the choice: every output is one fp32 accumulator over K in
+ * ascending order, rounded once.  Process-wide; not thread-safe against concurrent launches.
+ * Returns D3TOM_ERR_INVALID_ARG for other values. */
+int d3tom_set_pair_tiles(int width);
+
 /* Sec. 3.2.1, "Rank(S_j) <= (1-alpha)|V|": number of kept tokens for keep
  * ratio r = 1-alpha.  Host arithmetic: clamp(floor(r*n_visual + 1e-9), 1, n_visual). */
 int d3tom_keep_count(int n_visual, double keep_ratio);

@@ -9,6 +9,7 @@
 #include "common.cuh"
 
 int g_d3tom_launch_overlap = 1;
+int g_d3tom_pair_tiles = -1;
 
 namespace {
 
@@ -193,6 +194,12 @@ int d3tom_set_reference_kernels(d3tom_ctx* ctx, int on) {
 
 int d3tom_set_launch_overlap(int on) {
   g_d3tom_launch_overlap = on ? 1 : 0;
+  return D3TOM_OK;
+}
+
+int d3tom_set_pair_tiles(int width) {
+  if (width != -1 && width != 0 && width != 256) return D3TOM_ERR_INVALID_ARG;
+  g_d3tom_pair_tiles = width;
   return D3TOM_OK;
 }
 

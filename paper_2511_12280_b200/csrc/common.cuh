@@ -69,6 +69,7 @@ __device__ __forceinline__ void grid_dependency_enter() {
 
 // Process-wide switch behind d3tom_set_launch_overlap (1 = overlap, the default).
 extern int g_d3tom_launch_overlap;
+extern int g_d3tom_pair_tiles;      // dense layers on CTA pairs: -1 chosen per shape, 0 never, 256 wherever the shape allows
 
 template <typename... Params, typename... Args>
 inline cudaError_t launch_serialized(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,

@@ -528,6 +528,224 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (warp == 2) ptx::tmem_dealloc(tmem_base, 2 * S::kAccStride);
 }
 
+// ---------------------------------------------------------------- CTA pairs
+// Two CTAs of a cluster (ranks 0 and 1, neighbouring SMs) compute one 256 x BN tile with `cta_group::2` MMAs: each CTA
+// holds its own 128 rows of A and HALF of the B tile (BN / 2 rows) in shared memory, the tensor cores of both read both
+// halves, and each CTA's 128 x BN accumulator lands in its own tensor memory.  Per k-block a CTA pulls 16 + BN / 4 KB out
+// of L2 instead of 16 + BN / 2 KB: 32 KB for 512 tensor cycles at BN = 256, where the single-CTA 128 x 256 tile needs 48 KB
+// and is bound by what an SM can pull out of L2 (about 56 B per cycle).
+//   * both CTAs run the same warp roles; each loader thread waits on its OWN `empty` barrier and loads its own boxes, whose
+//     bytes are counted on rank 0's `full` barrier (rank 0's loader threads expect the bytes of both CTAs);
+//   * one thread of rank 0 issues every MMA and commits to the `empty` / `acc_full` barriers of BOTH CTAs;
+//   * the epilogue warps of both CTAs arrive on rank 0's `acc_empty` barrier (8 arrivals);
+//   * before a CTA leaves, its loaders have seen every commit aimed at it, rank 0 has seen every epilogue arrival, and
+//     the two CTAs meet in a cluster barrier; tensor memory is allocated and freed by warp 2 of both CTAs together.
+// Whole tiles only (no K split); every mbarrier wait is bounded as elsewhere.
+template <int BN> struct PairSmem {
+  static constexpr int kABytes = kBM * kBK * 2, kBBytes = (BN / 2) * kBK * 2;
+  static constexpr int kStages = 6;
+  static constexpr int kBytes = kStages * (kABytes + kBBytes) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
+  static_assert(BN % 32 == 0 && BN <= 256 && (BN / 2) % 8 == 0, "half of the B tile is a whole number of 8-row swizzle groups");
+  static_assert(EPI != kEpiSim, "the dense layers only");
+  using S = PairSmem<BN>;
+  constexpr int kStages = S::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a_s = smem;
+  uint8_t* b_s = smem + kStages * S::kABytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * (S::kABytes + S::kBBytes));
+  uint64_t* empty = full + kStages;
+  uint64_t* acc_full = empty + kStages;       // [2]
+  uint64_t* acc_empty = acc_full + 2;         // [2] (rank 0's are the ones in use)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const bool leader = rank == 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }   // A and B loaders of rank 0; one commit
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&acc_full[i], 1); ptx::mbar_init(&acc_empty[i], 8); }   // four epilogue warps in each CTA
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 2) { ptx::tmem_alloc_pair(tmem_slot, 512); ptx::tmem_relinquish_pair(); }
+  grid_dependency_wait();
+  grid_dependency_release();
+  ptx::tc_fence_before_sync();
+  ptx::cluster_sync();                     // the peer's barriers exist before anything arrives on them
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const int tiles = p.m_tiles * p.n_tiles;
+  const int n_pairs = gridDim.x >> 1, pair = blockIdx.x >> 1;
+  // tile t: M fastest, so that the pairs of a round share their B tiles in L2
+  auto tile_m0 = [&](int t) { return (t % p.m_tiles) * (2 * kBM); };
+  auto tile_n0 = [&](int t) { return (t / p.m_tiles) * (EPI == kEpiGateUp ? BN / 2 : BN); };
+
+  if (warp == 0 || warp == 6) {
+    // ------------------------------------------------------------ TMA producers: warp 0 streams A, warp 6 streams B
+    if (lane == 0) {
+      const bool is_a = warp == 0;
+      const CUtensorMap* tm = is_a ? &tmap_a : &tmap_b;
+      uint8_t* ring = is_a ? a_s : b_s;
+      const int stage_bytes = is_a ? S::kABytes : S::kBBytes;
+      ptx::prefetch_tensormap(tm);
+      int it = 0;
+      bool ok = true;
+      for (int t = pair; t < tiles && ok; t += n_pairs) {
+        const int n0 = tile_n0(t);
+        // this CTA's rows: its half of the 256 rows of A; its half of the B tile (gate rows for rank 0, up rows for rank 1)
+        const int row0 = is_a ? tile_m0(t) + (int)rank * kBM
+                              : (EPI == kEpiGateUp ? (leader ? n0 : p.up_row_offset + n0) : n0 + (int)rank * (BN / 2));
+        for (int kbk = 0; kbk < p.num_k_blocks; ++kbk, ++it) {
+          const int s = it % kStages;
+          ok = ptx::mbar_wait(&empty[s], ((it / kStages) & 1) ^ 1, abort_flag, p.dev_status);
+          if (!ok) break;
+          if (leader) ptx::mbar_arrive_expect_tx(&full[s], 2 * stage_bytes);     // this operand's boxes of both CTAs
+          ptx::tma_load_2d_pair(ring + s * stage_bytes, tm, &full[s], kbk * kBK, row0);
+        }
+      }
+      // every commit aimed at this CTA's `empty` barriers has landed before the CTA may leave
+      for (int j = it > kStages ? it - kStages : 0; j < it && ok; ++j)
+        ok = ptx::mbar_wait(&empty[j % kStages], (j / kStages) & 1, abort_flag, p.dev_status);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (rank 0 only)
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(2 * kBM, BN, 0, 0);
+      const ptx::SmemDesc a_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(a_s));
+      const ptx::SmemDesc b_desc0 = ptx::smem_desc_kmajor_sw128(ptx::smem_u32(b_s));
+      int it = 0, lt = 0;
+      bool ok = true;
+      for (int t = pair; t < tiles && ok; t += n_pairs, ++lt) {
+        const int buf = lt & 1;
+        ok = ptx::mbar_wait(&acc_empty[buf], ((lt >> 1) & 1) ^ 1, abort_flag, p.dev_status);   // both epilogues done with it
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t tmem_acc = tmem_base + (uint32_t)buf * 256u;
+        for (int kbk = 0; kbk < p.num_k_blocks; ++kbk, ++it) {
+          const int s = it % kStages;
+          ok = ptx::mbar_wait(&full[s], (it / kStages) & 1, abort_flag, p.dev_status);
+          if (!ok) break;
+          ptx::tc_fence_after_sync();
+          const ptx::SmemDesc ad = ptx::smem_desc_advance(a_desc0, s * S::kABytes), bd = ptx::smem_desc_advance(b_desc0, s * S::kBBytes);
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk)
+            ptx::mma_ss_pair(tmem_acc, ptx::smem_desc_advance(ad, kk * 32), ptx::smem_desc_advance(bd, kk * 32), idesc,
+                             (kbk > 0 || kk > 0) ? 1u : 0u);
+          ptx::mma_commit_pair(&empty[s], 3);      // frees the stage in both CTAs once these MMAs have read it
+        }
+        if (ok) ptx::mma_commit_pair(&acc_full[buf], 3);
+      }
+      // the peer's epilogue arrivals for the last tiles have landed before this CTA may leave
+      for (int j = lt > 2 ? lt - 2 : 0; j < lt && ok; ++j)
+        ok = ptx::mbar_wait(&acc_empty[j & 1], (j >> 1) & 1, abort_flag, p.dev_status);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    int lt = 0;
+    for (int t = pair; t < tiles; t += n_pairs, ++lt) {
+      const int buf = lt & 1;
+      const bool ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[buf], (lt >> 1) & 1, abort_flag, p.dev_status));
+      if (!ok) break;
+      ptx::tc_fence_after_sync();
+      const uint32_t t_row = tmem_base + (uint32_t)buf * 256u + ((uint32_t)(quarter * 32) << 16);
+      const int grow = tile_m0(t) + (int)rank * kBM + row;
+      const int n0 = tile_n0(t);
+      if (EPI == kEpiProj) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_row + c, r);
+          ptx::tmem_wait_ld();
+          const int gcol = n0 + c, which = gcol / p.out_cols;
+          if (grow < p.out_rows && which < 3) {
+            __nv_bfloat16* dst = p.out[which] + (size_t)grow * p.out_cols + (gcol - which * p.out_cols);
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[i + 2 * j]), __uint_as_float(r[i + 2 * j + 1]));
+                w[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else if (EPI == kEpiLinear) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          ptx::tmem_ld32(t_row + c, r);
+          ptx::tmem_wait_ld();
+          if (grow < p.out_rows && n0 + c < p.ld_out) {
+            const size_t off = (size_t)grow * p.ld_out + n0 + c;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4] = {0u, 0u, 0u, 0u};
+              if (p.residual != nullptr) {
+                const uint4 rr = *reinterpret_cast<const uint4*>(p.residual + off + i);
+                w[0] = rr.x; w[1] = rr.y; w[2] = rr.z; w[3] = rr.w;
+              }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float lo = __uint_as_float(r[i + 2 * j]) + __uint_as_float(w[j] << 16);
+                const float hi = __uint_as_float(r[i + 2 * j + 1]) + __uint_as_float(w[j] & 0xffff0000u);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+                w[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(p.lin_out + off + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN / 2; c += 32) {
+          uint32_t g[32], up[32];
+          ptx::tmem_ld32(t_row + c, g);
+          ptx::tmem_ld32(t_row + BN / 2 + c, up);
+          ptx::tmem_wait_ld();
+          if (grow < p.out_rows) {
+            __nv_bfloat16* dst = p.lin_out + (size_t)grow * p.ld_out + n0 + c;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float g0 = __uint_as_float(g[i + 2 * j]), g1 = __uint_as_float(g[i + 2 * j + 1]);
+                const float a0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(up[i + 2 * j]);
+                const float a1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(up[i + 2 * j + 1]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(a0, a1);
+                w[j] = *reinterpret_cast<uint32_t*>(&h2);
+              }
+              *reinterpret_cast<uint4*>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      }
+      // the accumulator may be overwritten once the four warps of both CTAs have read it: tell rank 0
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) {
+        if (leader) ptx::mbar_arrive(&acc_empty[buf]);
+        else ptx::mbar_arrive_cluster(&acc_empty[buf], 0);
+      }
+    }
+  }
+  __syncwarp();                            // (the lanes that ran a role's loop rejoin their warp before the aligned barrier)
+  ptx::tc_fence_before_sync();
+  ptx::cluster_sync();                     // neither CTA frees tensor memory or leaves while the other may still reach it
+  if (warp == 2) ptx::tmem_dealloc_pair(tmem_base, 512);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -605,6 +823,49 @@ int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, Ge
   return D3TOM_OK;
 }
 
+// How many CTA pairs of this kernel the device holds at once (asked once per device).
+template <int BN, int EPI>
+int launch_gemm_pair(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t s) {
+  const long long tiles = (long long)p.m_tiles * p.n_tiles;
+  if (tiles <= 0) return D3TOM_OK;
+  auto kernel = gemm_pair_kernel<BN, EPI>;
+  D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem<BN>::kBytes));
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = g_d3tom_launch_overlap ? 1 : 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(ctx->sm_count & ~1)); cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = PairSmem<BN>::kBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
+  static int resident_pairs[64] = {};
+  int& pairs = resident_pairs[ctx->device & 63];
+  if (pairs == 0) {
+    int n = 0;
+    D3TOM_CUDA_TRY(ctx, cudaOccupancyMaxActiveClusters(&n, kernel, &cfg));
+    if (n <= 0) return D3TOM_ERR_UNSUPPORTED;
+    pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
+  }
+  cfg.gridDim = dim3((unsigned)(2 * (tiles < pairs ? tiles : pairs)));
+  D3TOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, kernel, ta, tb, p));
+  return D3TOM_OK;
+}
+
+// Whether a dense layer of `rows` x `ncols` outputs runs as 256 x 256 tiles on CTA pairs.  Measured against the
+// single-CTA shapes, alternating the two in one process (projection / output projection / feed-forward network at
+// D = 4096, m = 12288, us): 1216 rows 94 / 51 / 294 against 92 / 56 / 303, 1152 rows 98 / 59 / 297 against
+// 87 / 39 / 257, 2176 rows 147 / 56 / 453 against 156 / 62 / 480, 4288 rows 281 / 105 / 914 against 303 / 132 / 1076,
+// 7800 rows 543 / 212 / 1715 against 583 / 290 / 1988.  A round of 74 pair tiles costs what a round of 148 tiles of
+// 256 x 256 costs per flop (both run at the tensor rate the board's power limit allows), so short layers, which are
+// decided by how the tiles fill the last round, keep their shapes; from about two thousand rows on the pairs win on
+// every layer: half the operand traffic per SM leaves more of the power budget to the tensor cores.
+bool use_pair_tiles(const d3tom_ctx* ctx, int rows, int ncols) {
+  if (ncols % 256 != 0 || ctx->sm_count < 2) return false;
+  if (g_d3tom_pair_tiles == 0) return false;
+  if (g_d3tom_pair_tiles == 256) return true;
+  return rows >= 2048;
+}
+
 }  // namespace
 
 int make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
@@ -644,6 +905,12 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
+  if (use_pair_tiles(ctx, total, 3 * D)) {
+    r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 128);       // a CTA's half of the weight tile
+    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+    p.m_tiles = ceil_div(total, 2 * kBM); p.n_tiles = 3 * D / 256;
+    return launch_gemm_pair<256, kEpiProj>(ctx, ta, tb, p, s);
+  }
   if (const int w2 = two_m_tile_width(ctx, total, 3 * D, D % 32 == 0)) {
     r = make_tmap_bf16_2d(&ta, x, (uint64_t)total, (uint64_t)D, (uint64_t)D, 2 * kBM);
     if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, (uint32_t)w2);
@@ -681,6 +948,12 @@ int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* r
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
+  if (use_pair_tiles(ctx, rows, N)) {
+    r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, 128);
+    if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
+    p.m_tiles = ceil_div(rows, 2 * kBM); p.n_tiles = N / 256;
+    return launch_gemm_pair<256, kEpiLinear>(ctx, ta, tb, p, s);
+  }
   if (const int w2 = two_m_tile_width(ctx, rows, N, true)) {
     r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)K, (uint64_t)K, 2 * kBM);
     if (r == 0) r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, (uint32_t)w2);
@@ -709,6 +982,10 @@ int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int 
   p.lin_out = static_cast<__nv_bfloat16*>(act); p.ld_out = m; p.up_row_offset = m; p.out_rows = rows;
   p.dev_status = ctx->dev_status;
   p.m_tiles = ceil_div(rows, kBM); p.n_tiles = m / 128; p.batch = 1; p.k_splits = 1;
+  if (use_pair_tiles(ctx, rows, 2 * m)) {       // (the B map's box is already 128 rows: one CTA's half)
+    p.m_tiles = ceil_div(rows, 2 * kBM);
+    return launch_gemm_pair<256, kEpiGateUp>(ctx, ta, tb, p, s);
+  }
   {
     if (two_m_tile_width(ctx, rows, 2 * m, false) == 256) {
       r = make_tmap_bf16_2d(&ta, x, (uint64_t)rows, (uint64_t)D, (uint64_t)D, 2 * kBM);

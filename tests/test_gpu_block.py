@@ -68,6 +68,50 @@ def test_linear_and_ffn_bf16_shapes_that_take_256_row_tiles():
     run_linear(1216, 128, 12288, "bf16", residual=False, seed=9)
 
 
+def run_proj(rows, H, dh, seed=0):
+    dev = torch.device("cuda", 0)
+    D = H * dh
+    t = wl.block_inputs(seed, rows, D, 8, "bf16")
+    x = t["x"][:, :D].contiguous()
+    g = torch.Generator().manual_seed(seed + 1)
+    w = (torch.randn(3 * D, D, generator=g) * (4.0 / D ** 0.5)).to(torch.bfloat16)
+    ctx = B_.Context(max(rows, 1), 1, H, dh, 1, 1)
+    q, k, v = (torch.full((rows, D), float("nan"), dtype=torch.bfloat16, device=dev) for _ in range(3))
+    ctx.d3tom_proj_qkv(x.to(dev), w.to(dev), rows, D, q, k, v)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    want = orc.proj_qkv(pu.f64(x), pu.f64(w), H, "bf16")
+    for got, ref, name in zip((q, k, v), want, "qkv"):
+        pu.assert_close(pu.f64(got), ref.reshape(rows, D), "bf16", "%s of the projection, %d rows, D = %d" % (name, rows, D))
+    ctx.close()
+
+
+def test_dense_layers_on_cta_pairs():
+    # 256 x 256 tiles computed by two CTAs (each holds its 128 rows of x and half of the weight tile): a ragged last
+    # row tile whose second CTA has no rows at all, whole tiles, more tiles than pairs (several rounds); the output
+    # projection with and without residual and the gated feed-forward network (gate rows in one CTA, up rows in the other)
+    B_.d3tom_set_pair_tiles(256)
+    try:
+        run_proj(64, 4, 128)
+        run_proj(300, 4, 128, seed=1)
+        run_proj(1216, 8, 128, seed=2)
+        run_proj(5000, 2, 128, seed=3)
+        run_linear(300, 256, 512, "bf16", residual=True)
+        run_linear(129, 320, 256, "bf16", residual=True, in_place=True)
+        run_linear(2500, 192, 768, "bf16", residual=False)
+        run_ffn(300, 256, 512, "bf16", seed=5)
+        run_ffn(2300, 128, 384, "bf16", seed=6)
+    finally:
+        B_.d3tom_set_pair_tiles(-1)
+
+
+def test_long_dense_layers_take_cta_pairs_by_default():
+    # from about two thousand rows on the library picks the pair tiles itself
+    run_proj(2304, 4, 128, seed=7)
+    run_linear(2100, 256, 512, "bf16", residual=True, seed=8)
+    run_ffn(2100, 256, 256, "bf16", seed=9)
+
+
 def test_linear_fp32_odd_sizes():
     run_linear(70, 50, 45, "fp32", residual=True)
     run_linear(33, 7, 3, "fp32", residual=False)
