@@ -48,9 +48,10 @@ WORKLOAD_TEXT = {
           "one more decider per step, keep ratio 0.5 -> 0 (mean 0.25), 3 post-merge layers; a step = one denoising step",
     "C4": "C4: 8 ragged requests, 1024-4096 visual tokens each, 32 heads x 128, keep in {0.1,0.25,0.5}, 3 post-merge layers",
 }
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from the committed ncu
-# capture; null for configurations not captured, and null whenever attn_tc.cu has changed since the capture
-ATTN_TRAFFIC_BYTES = {"C2": 194.7e6}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel (the launch `roofline`
+# times: attention alone at the merge-layer length) from the committed ncu capture, mean of two launches; null for
+# configurations not captured, and null whenever attn_sk.cu / attn_tc.cu have changed since the capture
+ATTN_TRAFFIC_BYTES = {"C2": 177.0e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 REFERENCE_BUDGET_S = 240.0          # the CPU arm stops adding steps once they would not fit this
@@ -533,6 +534,9 @@ def measure_config(name, args, dev, local_rank, world, full):
         run()
         calls = {
             "attn_importance": lambda: step.attn_importance(q, k, v),
+            # the launch that `roofline` times: attention alone at the merge-layer length, no importance side-work
+            "attn_alone": lambda: step.ctx.d3tom_attn_varlen(q, k, v, step.cu_seqlens, step.nB, step.total,
+                                                             step.max_seqlen, step.scale, step.attn_out),
             "select": lambda: step.select(),
             "merge": lambda: step.merge(),
             "step": run,
@@ -720,7 +724,7 @@ def measure_config(name, args, dev, local_rank, world, full):
     # ---- roofline of the dominant kernel (merge-layer attention): 4 N^2 D flops per request
     attn_flops = sum(4.0 * n * n * step.D for n in step.seqlens_h)
     achieved = attn_flops / (attn_kernel_us * 1e-6) / 1e12
-    res["roofline"] = {"bound": "tensor", "kernel": "attn_tc_kernel (merge-layer attention, timed alone)",
+    res["roofline"] = {"bound": "tensor", "kernel": "attn_sk_kernel / attn_tc_kernel (merge-layer attention, timed alone; one request with uneven rounds takes the balanced walk)",
                        "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                        "frac": achieved / peaks["bf16_tflops"], "traffic": ATTN_TRAFFIC_BYTES.get(name),
                        "algorithmic_bytes": 4.0 * step.total * step.D * q.element_size(),
@@ -776,7 +780,7 @@ def main():
     ap.add_argument("--deciders", default="all", choices=["all", "recent"],
                     help="schedule config: every token revealed so far, or only those of the previous step")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
-    ap.add_argument("--only", default=None, choices=["attn_importance", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
+    ap.add_argument("--only", default=None, choices=["attn_importance", "attn_alone", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
                     help="profiling aid: after one full step, run just this call --steps times and exit")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
