@@ -823,12 +823,40 @@ int launch_gemm(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, Ge
   return D3TOM_OK;
 }
 
-// How many CTA pairs of this kernel the device holds at once (asked once per device).
+// How many CTA pairs of this kernel the device holds at once (asked once per device; 0 = clusters of two cannot be
+// launched here, and the caller keeps single-CTA tiles).
+template <int BN, int EPI>
+int resident_pairs(d3tom_ctx* ctx) {
+  static int cached[64] = {};
+  int& pairs = cached[ctx->device & 63];
+  if (pairs == 0) {
+    auto kernel = gemm_pair_kernel<BN, EPI>;
+    pairs = -1;
+    if (ctx->sm_count >= 2 &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem<BN>::kBytes) == cudaSuccess) {
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(ctx->sm_count & ~1)); cfg.blockDim = dim3(kGemmThreads);
+      cfg.dynamicSmemBytes = PairSmem<BN>::kBytes; cfg.attrs = attr; cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0)
+        pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
+    }
+    if (pairs < 0) (void)cudaGetLastError();     // (the refusal is not an error of the call in hand)
+  }
+  return pairs > 0 ? pairs : 0;
+}
+
 template <int BN, int EPI>
 int launch_gemm_pair(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& tb, GemmParams p, cudaStream_t s) {
   const long long tiles = (long long)p.m_tiles * p.n_tiles;
   if (tiles <= 0) return D3TOM_OK;
+  const int pairs = resident_pairs<BN, EPI>(ctx);
+  if (pairs <= 0) return D3TOM_ERR_UNSUPPORTED;
   auto kernel = gemm_pair_kernel<BN, EPI>;
+  // (the attribute belongs to the current device: set on every call, a process may drive several GPUs)
   D3TOM_CUDA_TRY(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PairSmem<BN>::kBytes));
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -836,17 +864,8 @@ int launch_gemm_pair(d3tom_ctx* ctx, const CUtensorMap& ta, const CUtensorMap& t
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = g_d3tom_launch_overlap ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(ctx->sm_count & ~1)); cfg.blockDim = dim3(kGemmThreads);
+  cfg.gridDim = dim3((unsigned)(2 * (tiles < pairs ? tiles : pairs))); cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = PairSmem<BN>::kBytes; cfg.stream = s; cfg.attrs = attr; cfg.numAttrs = 2;
-  static int resident_pairs[64] = {};
-  int& pairs = resident_pairs[ctx->device & 63];
-  if (pairs == 0) {
-    int n = 0;
-    D3TOM_CUDA_TRY(ctx, cudaOccupancyMaxActiveClusters(&n, kernel, &cfg));
-    if (n <= 0) return D3TOM_ERR_UNSUPPORTED;
-    pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
-  }
-  cfg.gridDim = dim3((unsigned)(2 * (tiles < pairs ? tiles : pairs)));
   D3TOM_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, kernel, ta, tb, p));
   return D3TOM_OK;
 }
@@ -905,7 +924,7 @@ int launch_proj_tc(d3tom_ctx* ctx, const void* x, const void* w, int total, int 
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  if (use_pair_tiles(ctx, total, 3 * D)) {
+  if (use_pair_tiles(ctx, total, 3 * D) && resident_pairs<256, kEpiProj>(ctx) > 0) {
     r = make_tmap_bf16_2d(&tb, w, (uint64_t)3 * D, (uint64_t)D, (uint64_t)D, 128);       // a CTA's half of the weight tile
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
     p.m_tiles = ceil_div(total, 2 * kBM); p.n_tiles = 3 * D / 256;
@@ -948,7 +967,7 @@ int launch_linear_tc(d3tom_ctx* ctx, const void* x, const void* w, const void* r
     const double cost = rounds * (cand == 256 ? 667.0 : cand == 192 ? 633.0 : 600.0);
     if (cost < best_cost) { best_cost = cost; bn = cand; }
   }
-  if (use_pair_tiles(ctx, rows, N)) {
+  if (use_pair_tiles(ctx, rows, N) && resident_pairs<256, kEpiLinear>(ctx) > 0) {
     r = make_tmap_bf16_2d(&tb, w, (uint64_t)N, (uint64_t)K, (uint64_t)K, 128);
     if (r != 0) { ctx->last_cuda_error = r; return D3TOM_ERR_CUDA; }
     p.m_tiles = ceil_div(rows, 2 * kBM); p.n_tiles = N / 256;
@@ -982,7 +1001,7 @@ int launch_gate_up_tc(d3tom_ctx* ctx, const void* x, const void* w_gate_up, int 
   p.lin_out = static_cast<__nv_bfloat16*>(act); p.ld_out = m; p.up_row_offset = m; p.out_rows = rows;
   p.dev_status = ctx->dev_status;
   p.m_tiles = ceil_div(rows, kBM); p.n_tiles = m / 128; p.batch = 1; p.k_splits = 1;
-  if (use_pair_tiles(ctx, rows, 2 * m)) {       // (the B map's box is already 128 rows: one CTA's half)
+  if (use_pair_tiles(ctx, rows, 2 * m) && resident_pairs<256, kEpiGateUp>(ctx) > 0) {       // (the B map's box is already 128 rows: one CTA's half)
     p.m_tiles = ceil_div(rows, 2 * kBM);
     return launch_gemm_pair<256, kEpiGateUp>(ctx, ta, tb, p, s);
   }
