@@ -407,6 +407,49 @@ def block_timings(step, w, w_post0, q, dev, timed, reps):
     return out
 
 
+def dense_ab(step, w, w_post, q, dev, reps=8, calls=6):
+    """Dense layers of a post-merge block on CTA pairs against single-CTA tiles, alternating the two shapes quickly so
+    that both see the same power state: median us per call of the projection, the output projection and the gated
+    feed-forward network at the shortened length N_m and at the full length N."""
+    import torch
+    from paper_2511_12280_b200 import binding as B_
+    from paper_2511_12280_b200 import workload as wl
+    D, m = step.D, 3 * step.D
+    t = wl.block_inputs(1000, 8, D, m, w.dtype)
+    w_o, w_gu, w_dn = t["w_o"].to(dev), t["w_gate_up"].to(dev), t["w_down"].to(dev)
+    ctx, out = step.ctx, {}
+    n_full, n_m = step.total, step.total_out
+    act = torch.empty(n_full, m, dtype=q.dtype, device=dev)
+    y = torch.empty(n_full, D, dtype=q.dtype, device=dev)
+    q3, k3, v3 = (torch.empty(n_full, D, dtype=q.dtype, device=dev) for _ in range(3))
+
+    def timed(fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(calls):
+            fn(i)
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / calls
+    try:
+        for tag, n, x in (("Nm", n_m, step.hidden_out), ("N", n_full, step.attn_out)):
+            fns = {"proj_qkv": lambda i: ctx.d3tom_proj_qkv(x, w_post[i % len(w_post)], n, D, q3, k3, v3),
+                   "proj_out": lambda i: ctx.d3tom_linear(x, w_o, x, n, D, D, y),
+                   "ffn": lambda i: ctx.d3tom_ffn(x, w_gu, w_dn, x, n, D, m, act, y)}
+            out[tag] = {"rows": n}
+            for name, fn in fns.items():
+                res = {0: [], 256: []}
+                for _ in range(reps):
+                    for width in (0, 256):
+                        B_.d3tom_set_pair_tiles(width)
+                        fn(0)
+                        res[width].append(timed(fn))
+                out[tag][name] = {"single_cta_us": float(np.median(res[0])), "cta_pairs_us": float(np.median(res[256]))}
+    finally:
+        B_.d3tom_set_pair_tiles(-1)
+    return out
+
+
 def make_kv_cache_case(step, w, k, v, dev):
     """Returns a callable that runs d3tom_merge_kv on the K/V rows of every request's [visual | prompt]
     prefix with the kept set that the step's select produced."""
@@ -558,6 +601,8 @@ def measure_config(name, args, dev, local_rank, world, full):
             calls["ffn"] = lambda: step.ctx.d3tom_ffn(step.hidden_out, w_gu, w_dn, step.hidden_out, step.total_out,
                                                       step.D, m_ff, act, y)
         torch.cuda.synchronize()
+        if args.only == "dense_ab":
+            return {"only": args.only, "config": name, "dense_ab": dense_ab(step, w, w_post, q, dev)}
         us = timed(calls[args.only], args.steps)
         return {"only": args.only, "us": us, "config": name}
 
@@ -780,7 +825,7 @@ def main():
     ap.add_argument("--deciders", default="all", choices=["all", "recent"],
                     help="schedule config: every token revealed so far, or only those of the previous step")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every kernel of a step from the host instead of replaying a CUDA graph")
-    ap.add_argument("--only", default=None, choices=["attn_importance", "attn_alone", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step"],
+    ap.add_argument("--only", default=None, choices=["attn_importance", "attn_alone", "select", "merge", "proj_qkv", "attn_varlen", "proj_out", "ffn", "step", "dense_ab"],
                     help="profiling aid: after one full step, run just this call --steps times and exit")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
