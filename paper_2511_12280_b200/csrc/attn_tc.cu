@@ -70,7 +70,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   constexpr int kTileBytes = S::kTileBytes;
   constexpr int kHalfBytes = kTile * 128;               // one 64-column sub-tile: 128 rows x 128 bytes
   constexpr int kHalves = DH / 64;
-  // CTAs are dispatched in the order of their index.  Per request: the first H work items take the
+  // CTAs are dispatched in the order of their index.  Requests of a batch go longest first (below).  Per request: the first H work items take the
   // LAST 256-row query block of every head (the response rows live there and decider rows do extra
   // work, so those CTAs must not end up in the last wave); the remaining items walk head by head
   // (one head's K/V stay hot in L2), query blocks from the end.  Items from `split_from` on are cut
@@ -78,7 +78,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   // wave, which then costs the time of a single tile instead of a pair.
   grid_dependency_enter();
   const int items = a.H * a.nqb, per_req = items + (items - a.split_from);
-  const int b = (int)blockIdx.x / per_req, lin = (int)blockIdx.x - b * per_req;
+  int b = (int)blockIdx.x / per_req;
+  const int lin = (int)blockIdx.x - b * per_req;
+  if (a.B > 1 && a.B <= 32) {
+    // Requests are dispatched longest first (a work item's time grows with its request's length, and the last wave
+    // should hold short items): the group of CTAs number b takes the request of rank b by descending length,
+    // ties by index.  Every warp works the ranks out for itself (one load per lane, B shuffles).
+    const int lane_ = threadIdx.x & 31;
+    const int nl = lane_ < a.B ? a.cu_seqlens[lane_ + 1] - a.cu_seqlens[lane_] : -1;
+    int rank = 0;
+    for (int o = 0; o < a.B; ++o) {
+      const int no = __shfl_sync(0xffffffffu, nl, o);
+      rank += (no > nl || (no == nl && o < lane_)) ? 1 : 0;
+    }
+    b = __ffs(__ballot_sync(0xffffffffu, lane_ < a.B && rank == b)) - 1;
+  }
   int item = lin, half = -1;
   if (lin >= a.split_from) { item = a.split_from + ((lin - a.split_from) >> 1); half = (lin - a.split_from) & 1; }
   int h, qb;
