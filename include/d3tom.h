@@ -124,6 +124,13 @@ int d3tom_set_launch_overlap(int on);
  * Returns D3TOM_ERR_INVALID_ARG for other values. */
 int d3tom_set_pair_tiles(int width);
 
+/* Which tensor-core attention kernel serves d3tom_attn_varlen / d3tom_attn_importance (Sec. 3.2.1): -1 (default) the
+ * library's choice per launch, 0 the kernels with two query tiles per CTA, 1 the kernel with one query tile per CTA and
+ * three score buffers wherever it supports the launch (bf16, head_dim 128, no importance side-work).  Results agree
+ * within the attention tolerance (different summation orders of the row sum).  Process-wide; not thread-safe against
+ * concurrent launches.  Returns D3TOM_ERR_INVALID_ARG for other values. */
+int d3tom_set_single_tile_attention(int mode);
+
 /* Sec. 3.2.1, "Rank(S_j) <= (1-alpha)|V|": number of kept tokens for keep
  * ratio r = 1-alpha.  Host arithmetic: clamp(floor(r*n_visual + 1e-9), 1, n_visual). */
 int d3tom_keep_count(int n_visual, double keep_ratio);

@@ -49,6 +49,7 @@ _SIGNATURES = {
     "d3tom_set_reference_kernels": (_I, [_P, _I]),
     "d3tom_set_launch_overlap": (_I, [_I]),
     "d3tom_set_pair_tiles": (_I, [_I]),
+    "d3tom_set_single_tile_attention": (_I, [_I]),
     "d3tom_keep_count": (_I, [_I, C.c_double]),
     "d3tom_schedule_alpha": (_I, [_I, _I, C.c_double, C.c_double, _I, C.POINTER(C.c_double)]),
     "d3tom_attn_importance": (_I, [_P, _I, _P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _I, _I, _F, _P, _P, _P, _P]),
@@ -127,6 +128,12 @@ def d3tom_set_pair_tiles(width: int):
     """Tile shape of the dense layers: -1 chosen per shape (default), 0 single-CTA tiles only, 256 forces
     256 x 256 tiles computed by CTA pairs wherever the layer's width allows."""
     _check(load().d3tom_set_pair_tiles(int(width)), "d3tom_set_pair_tiles")
+
+
+def d3tom_set_single_tile_attention(mode: int):
+    """Attention kernel choice: -1 per launch (default), 0 two query tiles per CTA, 1 one query tile per CTA with three
+    score buffers wherever supported (bf16, head_dim 128, no importance)."""
+    _check(load().d3tom_set_single_tile_attention(int(mode)), "d3tom_set_single_tile_attention")
 
 
 def d3tom_schedule_alpha(step: int, T: int, a_min: float, a_max: float, reversed_: bool = False) -> float:

@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libd3tom.so")
 OBJ_DIR = os.path.join(HERE, "_build")
-SOURCES = ["api.cu", "attn_simt.cu", "attn_tc.cu", "attn_sk.cu", "select.cu", "merge.cu", "merge_stream.cu", "proj_simt.cu", "gemm_tc.cu", "no_alloc.cu", "selftest.cu"]
+SOURCES = ["api.cu", "attn_simt.cu", "attn_tc.cu", "attn_sk.cu", "attn_one.cu", "select.cu", "merge.cu", "merge_stream.cu", "proj_simt.cu", "gemm_tc.cu", "no_alloc.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

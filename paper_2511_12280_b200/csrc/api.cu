@@ -10,6 +10,7 @@
 
 int g_d3tom_launch_overlap = 1;
 int g_d3tom_pair_tiles = -1;
+int g_d3tom_single_tile_attention = -1;
 
 namespace {
 
@@ -197,6 +198,12 @@ int d3tom_set_launch_overlap(int on) {
   return D3TOM_OK;
 }
 
+int d3tom_set_single_tile_attention(int mode) {
+  if (mode < -1 || mode > 1) return D3TOM_ERR_INVALID_ARG;
+  g_d3tom_single_tile_attention = mode;
+  return D3TOM_OK;
+}
+
 int d3tom_set_pair_tiles(int width) {
   if (width != -1 && width != 0 && width != 256) return D3TOM_ERR_INVALID_ARG;
   g_d3tom_pair_tiles = width;
@@ -258,7 +265,9 @@ static int attn_common(d3tom_ctx* ctx, d3tom_dtype dt, const void* q, const void
   a.max_deciders = ctx->lim.max_deciders > 0 ? ctx->lim.max_deciders : 1; a.vis_stride = ctx->vis_stride;
   a.dev_status = ctx->dev_status;
   if (dt == D3TOM_BF16 && !ctx->reference_kernels) {
-    st = launch_attn_sk(ctx, a, stream);                       // one request whose items do not fill whole rounds of SMs
+    st = D3TOM_ERR_UNSUPPORTED;
+    if (g_d3tom_single_tile_attention == 1) st = launch_attn_one(ctx, a, stream);   // one query tile per CTA
+    if (st == D3TOM_ERR_UNSUPPORTED) st = launch_attn_sk(ctx, a, stream);   // one request whose items do not fill whole rounds of SMs
     if (st == D3TOM_ERR_UNSUPPORTED) st = launch_attn_tc(ctx, a, stream);
   } else {
     st = launch_attn_simt(ctx, dt, a, stream);

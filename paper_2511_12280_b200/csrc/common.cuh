@@ -69,6 +69,7 @@ __device__ __forceinline__ void grid_dependency_enter() {
 
 // Process-wide switch behind d3tom_set_launch_overlap (1 = overlap, the default).
 extern int g_d3tom_launch_overlap;
+extern int g_d3tom_single_tile_attention;   // -1 chosen per launch, 0 never, 1 wherever the kernel supports the launch
 extern int g_d3tom_pair_tiles;      // dense layers on CTA pairs: -1 chosen per shape, 0 never, 256 wherever the shape allows
 
 template <typename... Params, typename... Args>
@@ -163,6 +164,7 @@ struct AttnArgs {
 int launch_attn_simt(d3tom_ctx* ctx, d3tom_dtype dt, const AttnArgs& a, cudaStream_t s);
 int launch_attn_tc(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s);
 int launch_attn_sk(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s);      // one request, work balanced over the SMs
+int launch_attn_one(d3tom_ctx* ctx, const AttnArgs& a, cudaStream_t s);     // one query tile per CTA, three score buffers
 int launch_importance_finish(d3tom_ctx* ctx, const AttnArgs& a, int max_visual, float* importance,
                              const int32_t* cu_vis, cudaStream_t s);
 int launch_select(d3tom_ctx* ctx, const float* importance, const int32_t* cu_vis, const int32_t* keep_count,

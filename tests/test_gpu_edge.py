@@ -119,6 +119,45 @@ def test_few_similarity_tiles_are_cut_along_k_and_every_slice_reduces_its_column
     pu.check_step(w, mode=B_.AGG_SUM, full_attention=False, n_sample_rows=24)
 
 
+def run_attention_only(lens, H, seed=0):
+    """d3tom_attn_varlen on random Q, K, V of a ragged batch against the oracle, every row."""
+    dev = torch.device("cuda", 0)
+    dh, total = 128, int(sum(lens))
+    g = torch.Generator().manual_seed(seed)
+    q, k, v = (torch.randn(total, H * dh, generator=g).to(torch.bfloat16) for _ in range(3))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    ctx = B_.Context(total, len(lens), H, dh, 1, max(lens))
+    out = torch.full((total, H * dh), float("nan"), dtype=torch.bfloat16, device=dev)
+    scale = 1.0 / dh ** 0.5
+    ctx.d3tom_attn_varlen(q.to(dev), k.to(dev), v.to(dev), torch.from_numpy(cu).to(dev), len(lens), total, max(lens), scale, out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    want = orc.round_storage(orc.attention(pu.f64(q).reshape(total, H, dh), pu.f64(k).reshape(total, H, dh),
+                                           pu.f64(v).reshape(total, H, dh), cu, scale), "bf16")
+    got = pu.f64(out)
+    assert np.isfinite(got).all()
+    pu.assert_close(got, want.reshape(total, H * dh), "bf16", "attention, one query tile per CTA, lengths %s" % (lens,))
+    ctx.close()
+
+
+def test_attention_with_one_query_tile_per_cta():
+    # the kernel with three score buffers: one key block only (the second warpgroup has nothing to do), two, three, four
+    # (the buffers come round), ragged last blocks, one-row requests, a batch of unequal lengths (longest first), and a
+    # whole step whose post-merge layer runs on it
+    B_.d3tom_set_single_tile_attention(1)
+    try:
+        run_attention_only([100], 2)
+        run_attention_only([128], 2, seed=1)
+        run_attention_only([129], 2, seed=2)
+        run_attention_only([300], 3, seed=3)
+        run_attention_only([513], 2, seed=4)
+        run_attention_only([1216], 4, seed=5)
+        run_attention_only([1, 700, 64, 257, 1000], 2, seed=6)
+        pu.check_step(small())
+    finally:
+        B_.d3tom_set_single_tile_attention(-1)
+
+
 def test_text_only_request_inside_a_batch():
     # a request without visual tokens between two ordinary ones: nothing to select or merge there, its rows are
     # copied, its attention runs as usual
